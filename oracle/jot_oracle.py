@@ -1,0 +1,228 @@
+"""CPU oracle for JoT token-level early stopping -- TEST INFRASTRUCTURE ONLY.
+
+A plain, slow restatement of the method in the paper's own order and notation
+(Section 4.1 and Algorithm 1 of "Just on Time: Token-Level Early Stopping for
+Diffusion Language Models").  It shares no code with the CUDA library, is never
+imported by it, and exists only so that tests, the smoke check and the
+benchmark's CPU-baseline leg have something independent to compare against.
+
+All floating point is float64.  Where floating point decides an integer (the
+test r >= tau of Eq. 8), both operands are first rounded to float32 -- the
+precision the device kernel takes the decision in -- and `near_margin` reports
+the positions whose decision is within 1e-3 (relative) of flipping.
+
+Readings taken where the paper is silent (each is a keyword argument so the
+choice is visible at the call site):
+  * the mask token itself is not a candidate prediction (`exclude_mask_token`);
+  * argmax ties resolve to the lowest token id; on an exact tie of the two
+    largest logits p2 = p1;
+  * the window sum of Eq. 5 skips j = i (i is masked) and positions outside the
+    canvas contribute nothing; w_max is not adjusted at the canvas edges;
+  * the transfer schedule is "k highest max-probability positions", with k from
+    a fixed per-block table, and it ranks ALL currently masked candidates; its
+    mask is OR-ed with the early-exit mask (Section 4.2 "Implementation
+    details"); `schedule_after_exit=True` gives the other reading of
+    Algorithm 1 (schedule ranks only what early exit left masked);
+  * in block mode candidates are restricted to the current block while the
+    spatial window still sees the whole canvas.
+
+Parity unpinned: the choice among those readings (no printed output of the
+paper distinguishes them).
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Callable, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+@dataclasses.dataclass(frozen=True)
+class JotParams:
+    """tau_max, tau_min, gamma, D of Algorithm 1; eps of Eq. 4 (1e-12, Section 4.2)."""
+    tau_max: float = 90.0
+    tau_min: float = 1.0
+    gamma: float = 0.5
+    D: int = 8
+    eps: float = 1e-12
+
+
+DREAM_DEFAULT = JotParams(90.0, 1.0, 0.5, 8)   # Table 1 caption
+LLADA_DEFAULT = JotParams(30.0, 1.0, 0.5, 8)   # Table 1 caption
+
+
+# ----------------------------------------------------------------------------
+# Eq. 4: confidence ratio from one row of logits
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass
+class RowStats:
+    m1: float      # largest logit
+    i1: int        # its index (lowest index among maxima)
+    m2: float      # second-largest logit as an order statistic (== m1 on an exact tie)
+    S: float       # sum_v exp(l_v - m1)
+
+    @property
+    def p1(self) -> float:
+        return 1.0 / self.S
+
+    @property
+    def p2(self) -> float:
+        return math.exp(self.m2 - self.m1) / self.S
+
+
+def row_stats(logits: np.ndarray, mask_id: Optional[int] = None) -> RowStats:
+    """Softmax without temperature over one row of logits; top-2 by a full sort (Section 4.1,
+    "Confidence Metric").  If mask_id is given that column is not a candidate."""
+    l = np.asarray(logits, dtype=np.float64).copy()
+    if mask_id is not None:
+        l[mask_id] = -np.inf
+    order = np.argsort(-l, kind="stable")      # stable: lowest index first among equals
+    i1 = int(order[0])
+    m1 = float(l[i1])
+    m2 = float(l[order[1]])
+    S = float(np.sum(np.exp(l - m1)))
+    return RowStats(m1, i1, m2, S)
+
+
+def confidence_ratio(p1: float, p2: float, eps: float = 1e-12) -> float:
+    """Eq. 4: r = p1 / (p2 + eps)."""
+    return p1 / (p2 + eps)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 5-7: spatial weight, softening factor, adaptive threshold
+# ----------------------------------------------------------------------------
+def w_max(gamma: float, D: int) -> float:
+    """Eq. 6 text: w_max = 2 * sum_{d=1..D} gamma^d."""
+    return 2.0 * sum(gamma ** d for d in range(1, D + 1))
+
+
+def spatial_weight(x: Sequence[int], i: int, mask_id: int, gamma: float, D: int) -> float:
+    """Eq. 5: sum of gamma^|i-j| over unmasked j with |i-j| <= D, written as the double loop it is.
+    j ranges over the whole canvas (prompt tokens count as unmasked)."""
+    w = 0.0
+    for j in range(len(x)):
+        if j == i:
+            continue
+        if abs(i - j) <= D and x[j] != mask_id:
+            w += gamma ** abs(i - j)
+    return w
+
+
+def softening(w: float, gamma: float, D: int) -> float:
+    """Eq. 6: phi = min(1, w / w_max)."""
+    return min(1.0, w / w_max(gamma, D))
+
+
+def threshold(phi: float, tau_max: float, tau_min: float) -> float:
+    """Eq. 7: tau = tau_max - (tau_max - tau_min) * phi."""
+    return tau_max - (tau_max - tau_min) * phi
+
+
+def position_threshold(x: Sequence[int], i: int, mask_id: int, p: JotParams) -> float:
+    return threshold(softening(spatial_weight(x, i, mask_id, p.gamma, p.D), p.gamma, p.D),
+                     p.tau_max, p.tau_min)
+
+
+# ----------------------------------------------------------------------------
+# transfer schedule (Section 3.2; Section 4.2 "Interaction with transfer schedules")
+# ----------------------------------------------------------------------------
+def transfer_counts(block_len: int, steps_per_block: int) -> List[int]:
+    """How many positions the schedule reveals at each step of a block: block_len spread evenly over
+    the steps, the remainder going to the earliest steps."""
+    base, rem = divmod(block_len, steps_per_block)
+    return [base + (1 if s < rem else 0) for s in range(steps_per_block)]
+
+
+# ----------------------------------------------------------------------------
+# one acceptance / freeze update (inner part of Algorithm 1)
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass
+class StepReport:
+    exited: List[int]          # E: positions finalised by the early-exit test
+    scheduled: List[int]       # U: positions chosen by the transfer schedule
+    near_margin: List[int]     # |r - tau| <= 1e-3 * tau : decision may legitimately differ in fp32
+    ratio: dict                # position -> r
+    tau: dict                  # position -> tau
+
+
+def accept_freeze(x: List[int], stats: dict, p: JotParams, mask_id: int, blk_lo: int, blk_hi: int,
+                  k_transfer: int, schedule_after_exit: bool = False) -> StepReport:
+    """Update one sequence in place.  `stats[i]` is a RowStats for every masked i in [blk_lo, blk_hi).
+
+    All decisions use the canvas and the statistics as they were at the start of the step.
+    """
+    x0 = list(x)
+    A = [i for i in range(blk_lo, blk_hi) if x0[i] == mask_id]          # Algorithm 1: M_n (in block)
+    ratio, tau, near = {}, {}, []
+    E = []
+    for i in A:
+        st = stats[i]
+        r = confidence_ratio(st.p1, st.p2, p.eps)                         # Eq. 4
+        t = position_threshold(x0, i, mask_id, p)                         # Eq. 5-7
+        ratio[i], tau[i] = r, t
+        if abs(r - t) <= 1e-3 * abs(t):
+            near.append(i)
+        if np.float32(r) >= np.float32(t):                                # Eq. 8, decided in float32
+            E.append(i)
+    cand = [i for i in A if i not in E] if schedule_after_exit else A
+    k = min(k_transfer, len(cand))
+    ranked = sorted(cand, key=lambda i: (-stats[i].p1, i))                # highest max-prob, ties -> lower i
+    U = sorted(ranked[:k])
+    for i in set(E) | set(U):                                             # logical OR, uncapped
+        x[i] = stats[i].i1                                                # finalise by argmax
+    return StepReport(E, U, near, ratio, tau)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 1 (with semi-autoregressive blocks for block_len < gen_len)
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass
+class Trajectory:
+    x: List[int]
+    steps_used: int
+    canvases: List[List[int]]        # canvas BEFORE each step that ran
+    reports: List[StepReport]
+    exit_step: List[int]             # per position: 1-based step that finalised it, 0 if never masked
+    blocks: List[Tuple[int, int]]    # (blk_lo, blk_hi) of each step that ran
+
+
+def generate(logits_fn: Callable[[List[int], List[int]], dict], prompt: Sequence[int], gen_len: int,
+             steps: int, p: JotParams, mask_id: int, block_len: Optional[int] = None,
+             exclude_mask_token: bool = True, schedule_after_exit: bool = False,
+             stats_fn: Optional[Callable[[List[int], List[int]], dict]] = None) -> Trajectory:
+    """Algorithm 1 for one sequence.
+
+    logits_fn(x, rows) returns {i: logits row (length K)} for the requested masked positions;
+    alternatively stats_fn(x, rows) returns {i: RowStats} directly (for stub models in tests).
+    """
+    P = len(prompt)
+    Lb = gen_len if block_len is None else block_len
+    assert gen_len % Lb == 0
+    nb = gen_len // Lb
+    assert steps % nb == 0
+    Tb = steps // nb
+    ks = transfer_counts(Lb, Tb)
+    x = list(prompt) + [mask_id] * gen_len                                # initialise canvas
+    traj = Trajectory(x, 0, [], [], [0] * (P + gen_len), [])
+    for blk in range(nb):
+        lo, hi = P + blk * Lb, P + (blk + 1) * Lb
+        for s in range(Tb):
+            A = [i for i in range(lo, hi) if x[i] == mask_id]             # M_n
+            if not A:                                                     # break when nothing is masked
+                break
+            if stats_fn is not None:
+                stats = stats_fn(x, A)
+            else:
+                rows = logits_fn(x, A)
+                stats = {i: row_stats(rows[i], mask_id if exclude_mask_token else None) for i in A}
+            traj.canvases.append(list(x))
+            traj.blocks.append((lo, hi))
+            rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[s], schedule_after_exit)
+            traj.reports.append(rep)
+            traj.steps_used += 1
+            for i in set(rep.exited) | set(rep.scheduled):
+                traj.exit_step[i] = traj.steps_used
+        assert all(x[i] != mask_id for i in range(lo, hi)), "block not finished within its steps"
+    return traj

@@ -1,0 +1,284 @@
+"""Pins for the acceptance side of the CPU oracle (Section 4.1, Algorithm 1) against what the paper and
+plain mathematics fix: printed constants, hand-worked closed forms, brute force, invariants."""
+import math
+import random
+
+import numpy as np
+import pytest
+
+from conftest import read_table
+from oracle import jot_oracle as jo
+
+M = 99  # a mask id for toy canvases
+
+
+def canvas(pattern):
+    """'r' resolved, 'm' masked."""
+    return [M if c == "m" else 7 for c in pattern]
+
+
+# ---------------------------------------------------------------- Eq. 5-7: printed / hand-worked values
+def test_w_max_closed_forms():
+    for gamma, D, want in read_table("w_max.txt"):
+        assert jo.w_max(gamma, int(D)) == pytest.approx(want, rel=1e-9)
+    assert jo.w_max(0.5, 8) == 255.0 / 128.0
+
+
+def test_threshold_table_next_to_prompt():
+    x = canvas("r" * 12 + "m" * 40)
+    for k, w, phi, t90, t30 in read_table("threshold_table.txt"):
+        i = 11 + int(k)
+        assert jo.spatial_weight(x, i, M, 0.5, 8) == pytest.approx(w, abs=1e-15)
+        assert jo.softening(w, 0.5, 8) == pytest.approx(phi, rel=1e-14, abs=1e-16)
+        assert jo.position_threshold(x, i, M, jo.DREAM_DEFAULT) == pytest.approx(t90, rel=1e-14)
+        assert jo.position_threshold(x, i, M, jo.LLADA_DEFAULT) == pytest.approx(t30, rel=1e-14)
+
+
+def test_threshold_endpoints_and_single_neighbour():
+    # interior of a masked region keeps tau_max; fully resolved window gives tau_min (text after Eq. 7)
+    x = canvas("m" * 30)
+    assert jo.position_threshold(x, 15, M, jo.DREAM_DEFAULT) == 90.0
+    x = canvas("r" * 10 + "m" + "r" * 10)
+    assert jo.position_threshold(x, 10, M, jo.DREAM_DEFAULT) == pytest.approx(1.0, abs=1e-12)
+    # one resolved neighbour at distance 1 only: phi = 0.5 / (255/128) = 64/255
+    x = canvas("m" * 10 + "r" + "m" * 10)
+    assert jo.softening(jo.spatial_weight(x, 11, M, 0.5, 8), 0.5, 8) == pytest.approx(64 / 255)
+    assert jo.position_threshold(x, 11, M, jo.DREAM_DEFAULT) == pytest.approx(90 - 89 * 64 / 255)
+    assert jo.position_threshold(x, 9, M, jo.DREAM_DEFAULT) == pytest.approx(90 - 89 * 64 / 255)
+
+
+def test_window_radius_and_edges():
+    # a resolved token at distance D counts, at D+1 it does not; outside the canvas nothing counts
+    x = canvas("r" + "m" * 9)
+    assert jo.spatial_weight(x, 8, M, 0.5, 8) == 0.5 ** 8
+    assert jo.spatial_weight(x, 9, M, 0.5, 8) == 0.0
+    x = canvas("m" + "r" * 3)
+    assert jo.spatial_weight(x, 0, M, 0.5, 8) == 0.5 + 0.25 + 0.125
+    # asymmetric: the position itself (j = i) is never counted even when resolved elsewhere
+    x = canvas("rrmrr")
+    assert jo.spatial_weight(x, 2, M, 0.3, 1) == pytest.approx(0.6)
+
+
+def test_no_spatial_special_case():
+    # tau_max == tau_min: the threshold is the same everywhere (threshold-only ablation, Section 5.2)
+    p = jo.JotParams(90.0, 90.0, 0.5, 8)
+    x = canvas("rrrrmmmmmmmmrmmmrr")
+    assert {jo.position_threshold(x, i, M, p) for i in range(len(x)) if x[i] == M} == {90.0}
+
+
+def test_spatial_weight_is_a_1d_convolution():
+    # Section 4.2 "Computational overhead": the weight is a 1-D convolution with a fixed kernel
+    rng = random.Random(3)
+    for gamma, D in [(0.5, 8), (0.3, 8), (0.7, 8), (0.9, 16), (0.5, 4)]:
+        x = [M if rng.random() < 0.6 else 5 for _ in range(57)]
+        res = np.array([0.0 if t == M else 1.0 for t in x])
+        ker = np.array([gamma ** abs(d) if d != 0 else 0.0 for d in range(-D, D + 1)])
+        conv = np.convolve(res, ker, mode="same")
+        for i in range(len(x)):
+            if x[i] == M:
+                assert jo.spatial_weight(x, i, M, gamma, D) == pytest.approx(conv[i], rel=1e-12, abs=1e-15)
+                assert 0.0 <= jo.softening(conv[i], gamma, D) <= 1.0
+
+
+# ---------------------------------------------------------------- Eq. 4: confidence ratio
+def test_ratio_is_a_logit_margin():
+    # Section 4.1: r >= tau asks for a top-2 logit gap of ln(tau): "about 4.5 for tau = 90 and 3.4 for 30"
+    assert math.log(90) == pytest.approx(4.5, abs=0.01)
+    assert math.log(30) == pytest.approx(3.4, abs=0.01)
+    for tau in (90.0, 30.0):
+        for delta, expect in ((+1e-6, True), (-1e-6, False)):
+            l = np.full(50, -3.0)
+            l[17] = 2.0
+            l[31] = 2.0 - math.log(tau) - delta
+            st = jo.row_stats(l)
+            r = jo.confidence_ratio(st.p1, st.p2, 1e-12)
+            assert (r >= tau) == expect
+            assert r == pytest.approx(math.exp(st.m1 - st.m2), rel=1e-9)
+            assert st.i1 == 17
+
+
+def test_row_stats_brute_force_tiny_vocab():
+    rng = random.Random(0)
+    for trial in range(200):
+        V = rng.randint(3, 16)
+        l = [rng.choice([-2.0, -1.0, 0.0, 0.5, 1.0, 3.0]) + (rng.random() if trial % 2 else 0.0) for _ in range(V)]
+        mid = rng.randrange(V) if trial % 3 == 0 else None
+        st = jo.row_stats(np.array(l), mid)
+        cand = [(v, i) for i, v in enumerate(l) if i != mid]
+        z = sum(math.exp(v) for v, _ in cand)
+        probs = sorted(((math.exp(v) / z, i) for v, i in cand), key=lambda t: (-t[0], t[1]))
+        best = max(v for v, _ in cand)
+        assert st.i1 == min(i for v, i in cand if v == best)
+        assert st.p1 == pytest.approx(probs[0][0], rel=1e-12)
+        assert st.p2 == pytest.approx(probs[1][0], rel=1e-12)
+        assert st.p1 >= st.p2
+        if sum(1 for v, _ in cand if v == best) > 1:       # exact tie: p2 = p1, r < 1
+            assert st.m2 == st.m1
+            assert jo.confidence_ratio(st.p1, st.p2) < 1.0
+
+
+def test_ratio_temperature_invariance_of_the_definition():
+    # r uses un-tempered logits, so it is exp(gap) whatever else is in the row
+    l = np.array([0.3, 5.0, 1.0, -2.0])
+    st = jo.row_stats(l)
+    assert jo.confidence_ratio(st.p1, st.p2, 0.0) == pytest.approx(math.exp(4.0), rel=1e-12)
+
+
+def test_ratio_finite_when_p2_underflows():
+    l = np.array([0.0, 1000.0, -1000.0])
+    st = jo.row_stats(l)
+    r = jo.confidence_ratio(st.p1, st.p2, 1e-12)
+    assert math.isfinite(r) and r == pytest.approx(1e12, rel=1e-9)
+
+
+# ---------------------------------------------------------------- transfer schedule
+def test_transfer_counts():
+    assert jo.transfer_counts(64, 64) == [1] * 64
+    assert jo.transfer_counts(32, 32) == [1] * 32
+    assert jo.transfer_counts(10, 4) == [3, 3, 2, 2]
+    for L, T in [(256, 256), (7, 3), (5, 5), (3, 3), (100, 7)]:
+        ks = jo.transfer_counts(L, T)
+        assert sum(ks) == L and len(ks) == T and max(ks) - min(ks) <= 1
+
+
+# ---------------------------------------------------------------- accept / freeze on one step
+def stats_from_gap(i1, gap, p1=None):
+    """RowStats with a chosen top-2 gap; S chosen so p1 is as requested."""
+    S = (1.0 + math.exp(-gap)) if p1 is None else 1.0 / p1
+    return jo.RowStats(m1=1.0, i1=i1, m2=1.0 - gap, S=S)
+
+
+def test_accept_or_with_schedule_uncapped():
+    x = canvas("rrrr" + "mmmmmm")
+    lo, hi = 4, 10
+    # position 4 sits next to the prompt: tau = 90 - 89*phi with w = .5+.25+.125+.0625
+    stats = {i: stats_from_gap(100 + i, 0.1, p1=0.2) for i in range(lo, hi)}
+    stats[4] = stats_from_gap(104, math.log(20.0), p1=0.3)     # r = 20 >= tau(4)?
+    w4 = 0.5 + 0.25 + 0.125 + 0.0625
+    tau4 = 90 - 89 * w4 / (255 / 128)
+    assert tau4 == pytest.approx(90 - 89 * 8 / 17)          # 0.9375 / 1.9921875 = 8/17 -> 48.1176
+    stats[7] = stats_from_gap(107, 0.1, p1=0.9)                # schedule picks the max-prob row
+    rep = jo.accept_freeze(x, stats, jo.DREAM_DEFAULT, M, lo, hi, 1)
+    assert rep.exited == [] and rep.scheduled == [7]
+    assert x == [7, 7, 7, 7, M, M, M, 107, M, M]
+    # now make 4 clear its (softened) gate and 9 clear tau_max: both exit in the same step, plus schedule
+    x = canvas("rrrr" + "mmmmmm")
+    stats[4] = stats_from_gap(104, math.log(49.0), p1=0.3)
+    stats[9] = stats_from_gap(109, math.log(90.0) + 1e-9, p1=0.1)
+    rep = jo.accept_freeze(x, stats, jo.DREAM_DEFAULT, M, lo, hi, 1)
+    assert rep.exited == [4, 9] and rep.scheduled == [7]
+    assert x == [7, 7, 7, 7, 104, M, M, 107, M, 109]
+    # every position clears the gate: all finalised at once (Section 4.2 "uncapped")
+    x = canvas("rrrr" + "mmmmmm")
+    big = {i: stats_from_gap(200 + i, 10.0) for i in range(lo, hi)}
+    rep = jo.accept_freeze(x, big, jo.DREAM_DEFAULT, M, lo, hi, 1)
+    assert x == [7, 7, 7, 7, 204, 205, 206, 207, 208, 209] and len(rep.exited) == 6
+
+
+def test_schedule_ties_and_alternative_reading():
+    x = canvas("mmmm")
+    stats = {i: stats_from_gap(50 + i, 0.1, p1=0.5) for i in range(4)}
+    rep = jo.accept_freeze(x, stats, jo.JotParams(1e30, 1e30, 0.5, 8), M, 0, 4, 2)
+    assert rep.scheduled == [0, 1]                              # equal p1 -> lower positions
+    # OR reading: schedule ranks all of M_n, so it may coincide with an early exit ...
+    x = canvas("mmmm")
+    stats[2] = stats_from_gap(52, 20.0, p1=0.99)
+    rep = jo.accept_freeze(x, stats, jo.DREAM_DEFAULT, M, 0, 4, 1)
+    assert rep.exited == [2] and rep.scheduled == [2] and x.count(M) == 3
+    # ... while "schedule on the remaining positions" reveals one more
+    x = canvas("mmmm")
+    rep = jo.accept_freeze(x, stats, jo.DREAM_DEFAULT, M, 0, 4, 1, schedule_after_exit=True)
+    assert rep.exited == [2] and rep.scheduled == [0] and x.count(M) == 2
+
+
+def test_block_restriction_sees_full_canvas():
+    # candidates only inside [lo, hi); the window still sees resolved tokens outside the block
+    x = canvas("rrrr" + "mmmm" + "mmmm")
+    stats = {i: stats_from_gap(300 + i, 10.0) for i in range(4, 8)}
+    jo.accept_freeze(x, stats, jo.DREAM_DEFAULT, M, 4, 8, 1)
+    assert x[4:8] == [304, 305, 306, 307] and x[8:] == [M] * 4
+    p = jo.DREAM_DEFAULT
+    assert jo.position_threshold(x, 8, M, p) < 90.0            # neighbours in the earlier block count
+
+
+# ---------------------------------------------------------------- Algorithm 1: invariants + special cases
+def random_stats_fn(seed, V=1000, hot=0.3):
+    def fn(x, rows):
+        out = {}
+        for i in rows:
+            rng = random.Random(hash((seed, i, x.count(M))) & 0xFFFFFFFF)
+            gap = rng.random() * (8.0 if rng.random() < hot else 0.5)
+            out[i] = jo.RowStats(m1=2.0, i1=rng.randrange(V - 1), m2=2.0 - gap, S=1.0 + math.exp(-gap) + rng.random() * 3)
+        return out
+    return fn
+
+
+@pytest.mark.parametrize("block_len", [None, 8])
+@pytest.mark.parametrize("params", [jo.DREAM_DEFAULT, jo.LLADA_DEFAULT, jo.JotParams(60, 1, 0.7, 8), jo.JotParams(90, 30, 0.9, 16)])
+def test_generate_invariants(params, block_len):
+    rng = random.Random(1)
+    prompt = [rng.randrange(900) for _ in range(12)]
+    G, T = 32, 32
+    tr = jo.generate(None, prompt, G, T, params, M, block_len, stats_fn=random_stats_fn(5))
+    assert tr.x[:12] == prompt                                   # the prompt never changes
+    assert all(t != M for t in tr.x)                             # everything finalised
+    assert 1 <= tr.steps_used <= T
+    prev = None
+    for cv, rep in zip(tr.canvases, tr.reports):
+        if prev is not None:
+            assert cv.count(M) < prev.count(M)                   # at least one position per step
+            for a, b in zip(prev, cv):
+                assert a == M or a == b                          # frozen tokens never change
+        prev = cv
+    for a, b in zip(tr.canvases[-1], tr.x):
+        assert a == M or a == b
+    for i in range(12, 12 + G):                                  # exit_step agrees with the canvas history
+        s = tr.exit_step[i]
+        assert 1 <= s <= tr.steps_used
+        assert tr.canvases[s - 1][i] == M and (s == tr.steps_used or tr.canvases[s][i] != M)
+
+
+def test_generate_threshold_infinite_is_plain_topk_decoding():
+    # nothing clears the gate: exactly T steps of ordinary max-prob decoding (Section 4.2)
+    prompt = [1, 2, 3]
+    G = T = 10
+    fn = random_stats_fn(11)
+    tr = jo.generate(None, prompt, G, T, jo.JotParams(float("inf"), float("inf"), 0.5, 8), M, stats_fn=fn)
+    assert tr.steps_used == T and all(r.exited == [] for r in tr.reports)
+    x = prompt + [M] * G                                         # independent restatement of the baseline
+    for _ in range(T):
+        A = [i for i in range(len(x)) if x[i] == M]
+        st = fn(x, A)
+        best = min(A, key=lambda i: (-st[i].p1, i))
+        x[best] = st[best].i1
+    assert x == tr.x
+
+
+def test_generate_threshold_zero_finishes_one_step_per_block():
+    prompt = [1, 2, 3, 4]
+    tr = jo.generate(None, prompt, 32, 32, jo.JotParams(0.0, 0.0, 0.5, 8), M, None, stats_fn=random_stats_fn(2))
+    assert tr.steps_used == 1
+    tr = jo.generate(None, prompt, 32, 32, jo.JotParams(0.0, 0.0, 0.5, 8), M, 8, stats_fn=random_stats_fn(2))
+    assert tr.steps_used == 4
+    # step-speedup = configured / actual steps (Section 5.1)
+    assert 32 / tr.steps_used == 8.0
+
+
+def test_generate_with_logits_fn_excludes_mask_token():
+    V = 12
+    mid = V - 1
+
+    def logits_fn(x, rows):
+        out = {}
+        for i in rows:
+            l = np.linspace(-1, 1, V) * ((i % 3) - 1.0)
+            l[mid] = 50.0                                        # the model "predicts" the mask token
+            out[i] = l
+        return out
+    tr = jo.generate(logits_fn, [0, 1], 6, 6, jo.DREAM_DEFAULT, mid)
+    assert all(t != mid for t in tr.x)
+
+
+def test_reversal_budget_number():
+    # Section 5 (theory): 2 * 256 / (1 + 90) is "about 5.6"
+    assert 2 * 256 / 91 == pytest.approx(5.6, abs=0.05)
