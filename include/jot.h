@@ -1,0 +1,173 @@
+/*
+ * jot.h -- C ABI of the JoT denoising-step library for NVIDIA B200 (sm_100a).
+ *
+ * JoT ("Just on Time") is token-level early stopping for masked diffusion language models.  One
+ * denoising step is: a bidirectional transformer forward over the canvas (prompt followed by the
+ * generation region), the vocabulary-wide LM head reduced on the fly to per-position softmax
+ * statistics, the spatially adaptive acceptance test, and the in-place freeze/unmask update of
+ * the canvas.  Algorithm 1 of the paper is the loop around that step.
+ *
+ * Conventions for every entry point
+ *   - returns JOT_OK (0) or a negative jot_status; never throws, aborts or prints.
+ *   - "device" pointers are CUDA global-memory addresses on the current device, "host" pointers
+ *     are ordinary process memory.  Nothing is allocated on the device by the library except
+ *     where stated: the caller owns weights, workspace, inputs and outputs.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
+ *     enqueued on it; entry points that return host values synchronise that stream themselves.
+ *   - matrices are row-major; bf16 means the 16-bit brain-float storage format.
+ *   - all sequences of a batch have the same canvas length L (no padding, no ragged batches).
+ */
+#ifndef JOT_H_
+#define JOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    JOT_OK = 0,
+    JOT_ERR_ARG = -1,        /* null pointer, negative size, inconsistent ranges              */
+    JOT_ERR_SHAPE = -2,      /* geometry the kernels do not support (see each function)       */
+    JOT_ERR_WORKSPACE = -3,  /* workspace missing, misaligned or smaller than required        */
+    JOT_ERR_CUDA = -4,       /* a CUDA runtime/driver call failed: see jot_last_cuda_error()  */
+    JOT_ERR_TIMEOUT = -5,    /* a bounded device-side wait expired; outputs are undefined     */
+    JOT_ERR_DEVICE = -6      /* not an sm_100 device, or the driver lacks tensor-map support  */
+} jot_status;
+
+/* Static message for a status code. */
+const char* jot_status_string(int status);
+/* The cudaError_t (as int) behind the most recent JOT_ERR_CUDA on this thread, else 0. */
+int jot_last_cuda_error(void);
+
+/* Acceptance parameters: tau_max, tau_min, gamma, D of Algorithm 1 and epsilon of Eq. 4.
+ * Paper defaults (Table 1 caption; Section 4.2): (90, 1, 0.5, 8) for Dream, (30, 1, 0.5, 8) for
+ * LLaDA, eps = 1e-12.  1 <= D <= 32, 0 < gamma < 1 is what Eq. 5 assumes; gamma is not checked.
+ * schedule_after_exit = 0: the transfer schedule ranks all masked candidates and is OR-ed with the
+ * early-exit mask (Section 4.2 "Implementation details"); 1: it ranks only what early exit left. */
+typedef struct {
+    float tau_max, tau_min, gamma;
+    int32_t D;
+    float eps;
+    int32_t schedule_after_exit;
+} jot_params;
+
+/* Geometry of the denoiser f_theta (Algorithm 1 treats it as given).  Llama-style: RMSNorm,
+ * rotate-half RoPE on absolute canvas positions, grouped-query attention without any mask, SwiGLU
+ * MLP, untied LM head, no biases.  Supported: head_dim 64 or 128; d_model, d_ff and
+ * n_q_heads*head_dim multiples of 64; vocab a multiple of 8; n_q_heads a multiple of n_kv_heads. */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab, mask_id;
+    float rope_theta, rms_eps;
+} jot_model_config;
+
+/* bf16 device pointers, BORROWED for the model's lifetime and never written.
+ *   embed [vocab, d]; lm_head [vocab, d]; final_norm [d]
+ *   per layer l (arrays of n_layers host-resident pointers):
+ *     attn_norm[l] [d]; wqkv[l] [(nq + 2 nkv) * hd, d] (Q rows, K rows, V rows);
+ *     wo[l] [d, nq * hd]; mlp_norm[l] [d]; w_gate_up[l] [2 * d_ff, d] (gate rows, then up rows);
+ *     w_down[l] [d, d_ff].  Every pointer 16-byte aligned. */
+typedef struct {
+    const void* embed;
+    const void* lm_head;
+    const void* final_norm;
+    const void* const* attn_norm;
+    const void* const* wqkv;
+    const void* const* wo;
+    const void* const* mlp_norm;
+    const void* const* w_gate_up;
+    const void* const* w_down;
+} jot_weights;
+
+/* Generation settings of Algorithm 1.  gen_len = number of masked positions appended to the prompt;
+ * steps = T; block_len = semi-autoregressive block size (gen_len for a single block; must divide
+ * gen_len, and gen_len/block_len must divide steps).  exclude_mask_token != 0 keeps the mask token
+ * out of the candidate predictions. */
+typedef struct {
+    int32_t gen_len, steps, block_len;
+    int32_t exclude_mask_token;
+} jot_gen_config;
+
+typedef struct jot_model jot_model; /* opaque; host-side object owned by the library */
+
+/* Bytes of device workspace a model needs for batches up to max_batch sequences of canvas length up
+ * to max_seq.  Returns 0 on invalid arguments. */
+size_t jot_workspace_bytes(const jot_model_config* cfg, int max_batch, int max_seq);
+
+/* Create a model over borrowed weights and a caller-owned workspace (device, 1024-byte aligned, at
+ * least jot_workspace_bytes()).  Writes tables into the workspace (synchronous).  The workspace must
+ * stay alive and untouched by the caller until jot_free_model.  One model must not be used from two
+ * streams at once. */
+int jot_init_model(const jot_model_config* cfg, const jot_weights* weights, int max_batch, int max_seq,
+                   void* d_workspace, size_t workspace_bytes, jot_model** out);
+int jot_free_model(jot_model* m);
+
+/* Algorithm 1, "Compute logits" through "Compute confidence", for one step: the transformer forward
+ * over d_tokens [B, L] (int32, read-only), then the LM head over the rows that are masked
+ * (== mask_id) inside [blk_lo, blk_hi), reduced on the fly; logits are never stored.
+ * Outputs are device arrays indexed [B, L]; only entries of active rows are written:
+ *   top1_logit = largest logit, argmax = its token id (lowest id on ties), top2_logit = second
+ *   largest logit (equal to top1 on an exact tie), sumexp = sum_v exp(logit_v - top1_logit),
+ * so p1 = 1/sumexp and p2 = exp(top2 - top1)/sumexp (Section 4.1, "Confidence Metric").
+ * d_bump_id / d_bump_val ([B, L] int32 / float, both or neither NULL) add bump_val[b,i] to the logit
+ * of token bump_id[b,i] at position (b,i): a synthetic-workload hook.
+ * exclude_mask_token != 0 removes column mask_id from every statistic. */
+int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi,
+                     int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val,
+                     float* d_top1_logit, float* d_top2_logit, float* d_sumexp, int32_t* d_argmax,
+                     void* stream);
+
+/* The LM head + statistics part of jot_denoise_step alone, on caller-supplied final hidden states
+ * d_hidden [B*L, d] bf16 (already normalised).  Uses only lm_head, vocab, mask_id and d_model of
+ * the model.  Same outputs and options as jot_denoise_step. */
+int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_tokens, int B, int L,
+                      int blk_lo, int blk_hi, int exclude_mask_token, const int32_t* d_bump_id,
+                      const float* d_bump_val, float* d_top1_logit, float* d_top2_logit,
+                      float* d_sumexp, int32_t* d_argmax, void* stream);
+
+/* Section 4.1 Eq. 4-8 and the state update of Algorithm 1 for one step, in place on d_tokens [B, L].
+ * Candidates are the positions of [blk_lo, blk_hi) that hold mask_id.  For each: confidence ratio
+ * r = p1/(p2 + eps) from the statistics (Eq. 4), spatial weight over the whole canvas (Eq. 5,
+ * resolved = any position not holding mask_id, window radius D, positions outside the canvas
+ * contribute nothing), softening (Eq. 6), threshold (Eq. 7), test r >= tau in fp32 (Eq. 8).  The
+ * k_transfer candidates with the largest p1 (ties to the lower position) are chosen by the transfer
+ * schedule; a candidate chosen by either rule receives its argmax.  All decisions use the canvas as
+ * it was on entry.  params: one struct (host) applied to all sequences; per_seq_params must be 0
+ * here (per-sequence parameters are available through jot_generate).
+ * Outputs (device): d_n_masked [B] = candidates still masked after the update; optional
+ * d_exit_reason [B, L] uint8 (bit 0 early exit, bit 1 schedule; written for finalised positions
+ * only) and d_exit_step [B, L] int16 (= step_index, same positions). */
+int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask_id, int32_t* d_tokens,
+                      int B, int L, int blk_lo, int blk_hi, int k_transfer, const float* d_top1_logit,
+                      const float* d_top2_logit, const float* d_sumexp, const int32_t* d_argmax,
+                      int32_t* d_n_masked, uint8_t* d_exit_reason, int16_t* d_exit_step,
+                      int step_index, void* stream);
+
+/* Algorithm 1 for a batch of B independent sequences with prompts d_prompt [B, P] (int32, must not
+ * contain mask_id).  Each sequence keeps its own block pointer and step counter and idles once
+ * finished; the loop ends when no sequence has a masked position left, or after `steps` iterations.
+ * Outputs: d_out_tokens [B, P + gen_len] (device); h_steps_used [B] (host) = denoising steps each
+ * sequence actually ran (step speed-up = steps / steps_used, Section 5.1); optional
+ * h_forward_passes (host, one int) = batched forward passes executed.
+ * d_bump_id / d_bump_val: as in jot_denoise_step, indexed [B, P + gen_len], fixed across steps.
+ * Synchronises `stream` once per step to read the loop condition. */
+int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, const jot_gen_config* gen,
+                 const int32_t* d_prompt, int B, int P, const int32_t* d_bump_id, const float* d_bump_val,
+                 int32_t* d_out_tokens, int32_t* h_steps_used, int32_t* h_forward_passes, void* stream);
+
+/* C[M, N] (bf16) = A[M, K] (bf16) . W[N, K]^T (bf16) with fp32 accumulation on the tensor cores,
+ * optionally + residual[M, N] (bf16, may alias C).  The projection every layer of the forward is made
+ * of, exported for testing and benchmarking.  K and N multiples of 8; pointers 16-byte aligned.
+ * d_status: device int32 the kernel sets non-zero if a bounded wait expires (may be NULL). */
+int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
+                  int32_t* d_status, void* stream);
+
+/* Number of kernels this library has launched from the calling process so far. */
+int64_t jot_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JOT_H_ */

@@ -1,0 +1,351 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a:  D[M, N] = A[M, K] . W[N, K]^T, fp32 accumulate.
+//
+//   warp 0 (one lane)  TMA producer: 128 x 64 tile of A and BN x 64 tile of W per pipeline stage
+//   warp 1 (one lane)  tcgen05.mma issuer (UMMA 128 x BN x 16), accumulators in tensor memory,
+//                      two accumulator buffers so the epilogue of tile t overlaps the MMAs of tile t+1
+//   warps 2..5         epilogue: each thread owns one accumulator row (TMEM lane), reads it 32 columns
+//                      at a time and applies one of three epilogues:
+//        EPI_STORE   bf16(acc [+ residual])                                  -> C[M, N]
+//        EPI_SWIGLU  bf16(silu(gate) * up), gate/up from the two halves of W -> C[M, N/2]
+//        EPI_STATS   online (max, argmax, runner-up, sum-exp) per row over a range of vocabulary tiles;
+//                    the logits are never written (LM head of the denoising step)
+#pragma once
+#include "ptx.cuh"
+
+namespace jot {
+
+enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2 };
+
+constexpr int kBM = 128;          // rows per tile = TMEM lanes
+constexpr int kBK = 64;           // bf16 elements per 128-byte swizzled smem row
+constexpr int kGemmThreads = 192;
+
+struct GemmParams {
+    int M, N, K;                  // N = rows of W (for EPI_SWIGLU: 2 * d_ff)
+    __nv_bfloat16* C;             // EPI_STORE / EPI_SWIGLU output
+    const __nv_bfloat16* residual;  // EPI_STORE, nullable, same shape as C
+    int ldc;                      // row stride of C and residual, elements
+    int32_t* status;              // set non-zero when a bounded wait expired (nullable)
+    // EPI_STATS only
+    const int32_t* d_R;           // number of active rows (device)
+    const int32_t* rows;          // [R] flat canvas index b*L+i of each active row
+    const int32_t* bump_id;       // nullable, indexed by flat canvas index
+    const float* bump_val;
+    int mask_col;                 // column to exclude, or -1
+    float4* partials;             // [chunks][R_pad] (m1, bitcast i1, m2, S)
+    int R_pad;                    // row capacity of one chunk of partials (multiple of 128)
+};
+
+template <int BN>
+struct GemmSmem {
+    static constexpr int A_BYTES = kBM * kBK * 2;
+    static constexpr int B_BYTES = BN * kBK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (BN == 256) ? 4 : 6;
+    static constexpr int DYN_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align to 1024
+};
+
+// How the stats kernel splits the vocabulary: row blocks run side by side over the same vocabulary
+// range so that a tile of W fetched from HBM by one CTA is found in L2 by the others.
+__host__ __device__ inline void stats_partition(int R, int grid, int n_vt, int* n_rb, int* n_ch) {
+    int rb = (R + kBM - 1) / kBM;
+    int ch = rb > 0 ? grid / rb : 0;
+    if (ch > n_vt) ch = n_vt;
+    *n_rb = rb;
+    *n_ch = ch;
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB) {
+    using SM = GemmSmem<BN>;
+    constexpr int STAGES = SM::STAGES;
+    constexpr uint32_t TMEM_COLS = 2 * BN;                 // 256 or 512, a power of two
+    constexpr uint32_t IDESC = umma_idesc_bf16(kBM, BN);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = (p.K + kBK - 1) / kBK;
+
+    // ---- tile schedule (identical in every role) ----
+    int m_blk0 = 0, n_first = 0, n_count = 0;      // EPI_STATS: one row block, a range of vocabulary tiles
+    int num_m = (p.M + kBM - 1) / kBM;
+    constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
+    const int n_out = (EPI == EPI_SWIGLU) ? p.N / 2 : p.N;
+    const int num_n = (n_out + BN_OUT - 1) / BN_OUT;
+    int total_tiles = num_m * num_n;
+    int chunk = 0;
+    if (EPI == EPI_STATS) {
+        int R = *p.d_R, n_rb, n_ch;
+        stats_partition(R, gridDim.x, num_n, &n_rb, &n_ch);
+        chunk = n_rb > 0 ? blockIdx.x / n_rb : 0;
+        if (n_rb == 0 || chunk >= n_ch) {
+            n_count = 0;
+        } else {
+            m_blk0 = blockIdx.x % n_rb;
+            n_first = (int)((long long)chunk * num_n / n_ch);
+            n_count = (int)((long long)(chunk + 1) * num_n / n_ch) - n_first;
+        }
+        total_tiles = n_count;
+    }
+    auto tile_at = [&](int it, int& m_blk, int& n_blk) -> bool {
+        if (EPI == EPI_STATS) {
+            if (it >= total_tiles) return false;
+            m_blk = m_blk0;
+            n_blk = n_first + it;
+            return true;
+        }
+        int t = blockIdx.x + it * gridDim.x;
+        if (t >= total_tiles) return false;
+        m_blk = t % num_m;                        // row blocks fastest: neighbours share the W tile
+        n_blk = t / num_m;
+        return true;
+    };
+
+    // ---- setup ----
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 4);
+        }
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_base_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int m_blk, n_blk;
+            bool ok = true;
+            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
+                    uint8_t* sA = smem + stage * SM::STAGE_BYTES;
+                    uint8_t* sB = sA + SM::A_BYTES;
+                    mbar_arrive_expect_tx(&full_bar[stage], SM::STAGE_BYTES);
+                    tma_load_2d(sA, &tmA, &full_bar[stage], kb * kBK, m_blk * kBM);
+                    if (EPI == EPI_SWIGLU) {
+                        // gate rows, then the matching up rows: two boxes of BN/2 rows each
+                        tma_load_2d(sB, &tmB, &full_bar[stage], kb * kBK, n_blk * (BN / 2));
+                        tma_load_2d(sB + SM::B_BYTES / 2, &tmB, &full_bar[stage], kb * kBK,
+                                    p.N / 2 + n_blk * (BN / 2));
+                    } else {
+                        tma_load_2d(sB, &tmB, &full_bar[stage], kb * kBK, n_blk * BN);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            int m_blk, n_blk;
+            bool ok = true;
+            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abortp)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + stage * SM::STAGE_BYTES);
+                    const uint32_t b_addr = a_addr + SM::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        umma_bf16(d_tmem, umma_desc_k128(a_addr + k * 32), umma_desc_k128(b_addr + k * 32), IDESC,
+                                  (kb | k) != 0);
+                    }
+                    umma_commit(&empty_bar[stage]);       // smem stage reusable once these MMAs retire
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full[acc]);              // accumulator complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ================= epilogue (warps 2..5) =================
+        const int quad = warp & 3;                        // TMEM lanes [32*quad, 32*quad+32)
+        const int row_in_tile = quad * 32 + lane;
+        const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        int m_blk, n_blk;
+
+        // EPI_STATS running state of this thread's row
+        float m1 = -INFINITY, m2 = -INFINITY, S = 0.f;
+        int i1 = 0x7fffffff;
+        int bump_col = -1;
+        float bump_v = 0.f;
+        constexpr float L2E = 1.4426950408889634f;
+        if (EPI == EPI_STATS && total_tiles > 0) {
+            int R = *p.d_R;
+            int row = m_blk0 * kBM + row_in_tile;
+            if (row < R && p.bump_id != nullptr) {
+                int flat = p.rows[row];
+                bump_col = p.bump_id[flat];
+                bump_v = p.bump_val[flat];
+            }
+        }
+
+        bool ok = true;
+        for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+            if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t t_acc = lane_base + acc * BN;
+            const int row = m_blk * kBM + row_in_tile;
+
+            if (EPI == EPI_STORE) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    float v[32];
+                    tmem_ld32(t_acc + c * 32, v);
+                    tmem_ld_wait();
+                    const int col0 = n_blk * BN + c * 32;
+                    if (row < p.M) {
+                        __nv_bfloat16* dst = p.C + (size_t)row * p.ldc + col0;
+                        const __nv_bfloat16* res = p.residual ? p.residual + (size_t)row * p.ldc + col0 : nullptr;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            if (col0 + g * 8 < p.N) {         // N is a multiple of 8
+                                float x[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) x[j] = v[g * 8 + j];
+                                if (res) {
+                                    uint4 rv = *reinterpret_cast<const uint4*>(res + g * 8);
+                                    const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        float2 f = __bfloat1622float2(r2[j]);
+                                        x[2 * j] += f.x;
+                                        x[2 * j + 1] += f.y;
+                                    }
+                                }
+                                uint4 ov;
+                                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
+                                *reinterpret_cast<uint4*>(dst + g * 8) = ov;
+                            }
+                        }
+                    }
+                }
+            } else if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 64; ++c) {
+                    float g[32], u[32];
+                    tmem_ld32(t_acc + c * 32, g);
+                    tmem_ld32(t_acc + BN / 2 + c * 32, u);
+                    tmem_ld_wait();
+                    const int col0 = n_blk * (BN / 2) + c * 32;
+                    if (row < p.M) {
+                        __nv_bfloat16* dst = p.C + (size_t)row * p.ldc + col0;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (col0 + q * 8 < n_out) {
+                                uint4 ov;
+                                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    float g0 = g[q * 8 + 2 * j], g1 = g[q * 8 + 2 * j + 1];
+                                    float a0 = g0 / (1.f + __expf(-g0)) * u[q * 8 + 2 * j];
+                                    float a1 = g1 / (1.f + __expf(-g1)) * u[q * 8 + 2 * j + 1];
+                                    o2[j] = __floats2bfloat162_rn(a0, a1);
+                                }
+                                *reinterpret_cast<uint4*>(dst + q * 8) = ov;
+                            }
+                        }
+                    }
+                }
+            } else {
+                // ---- EPI_STATS: fold this tile's logits into (m1, i1, m2, S) ----
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    float v[32];
+                    tmem_ld32(t_acc + c * 32, v);
+                    tmem_ld_wait();
+                    const int col0 = n_blk * BN + c * 32;
+                    if (col0 >= p.N) break;                       // whole chunk past the vocabulary
+                    unsigned rel_b = (unsigned)(bump_col - col0);
+                    if (rel_b < 32u) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] += (j == (int)rel_b) ? bump_v : 0.f;
+                    }
+                    unsigned rel_m = (unsigned)(p.mask_col - col0);
+                    if (p.mask_col >= 0 && rel_m < 32u) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = (j == (int)rel_m) ? -INFINITY : v[j];
+                    }
+                    if (col0 + 32 > p.N) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = (col0 + j < p.N) ? v[j] : -INFINITY;
+                    }
+                    float cm = v[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+                    const float old_m = m1;
+                    if (cm > m2) {                                // only then can the top two change
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            float x = v[j];
+                            m2 = fmaxf(m2, fminf(x, m1));         // runner-up as an order statistic
+                            i1 = (x > m1) ? col0 + j : i1;        // strict: the lowest index wins ties
+                            m1 = fmaxf(m1, x);
+                        }
+                    }
+                    // S = sum exp(l - m1): rescale what was summed against the old maximum
+                    const float nm = m1 * L2E;
+                    float acc_s = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(v[j], L2E, -nm));
+                    S = S * ex2_approx(old_m * L2E - nm) + acc_s;
+                }
+            }
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+        if (EPI == EPI_STATS && ok && total_tiles > 0) {
+            p.partials[(size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile] =
+                make_float4(m1, __int_as_float(i1), m2, S);
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+    if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, 1);
+}
+
+}  // namespace jot

@@ -1,0 +1,203 @@
+// Bandwidth-bound pieces of the denoising step: embedding gather, RMSNorm (plain and with active-row
+// compaction), rotary embedding + V transpose, active-row list, merge of the LM-head partial
+// statistics, canvas initialisation.  All bf16 activations, fp32 arithmetic, 16-byte accesses.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "accept.cuh"
+
+namespace jot {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Block-wide sum for blockDim.x <= 1024 (result valid in every thread).
+__device__ __forceinline__ float block_sum(float v, float* scratch /* >= 33 floats */) {
+    v = warp_sum(v);
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+    if (l == 0) scratch[w] = v;
+    __syncthreads();
+    if (w == 0) {
+        float t = (l < nw) ? scratch[l] : 0.f;
+        t = warp_sum(t);
+        if (l == 0) scratch[32] = t;
+    }
+    __syncthreads();
+    float r = scratch[32];
+    __syncthreads();
+    return r;
+}
+
+// h[row, :] = E[tokens[row], :]          one CTA per row, 16-byte copies (d multiple of 8)
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E,
+                             __nv_bfloat16* __restrict__ h, int d) {
+    const int row = blockIdx.x;
+    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[row] * d);
+    uint4* dst = reinterpret_cast<uint4*>(h + (size_t)row * d);
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = src[i];
+}
+
+// out[r, :] = bf16( x[src_row, :] * rsqrt(mean(x^2) + eps) * gain ),  src_row = rows ? rows[r] : r.
+// With `rows`, only r < *d_R is processed (final norm + compaction of the active rows).
+// One CTA per output row; d multiple of 8 and d/8 <= 8 * blockDim.x.
+__global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
+                               __nv_bfloat16* __restrict__ out, int d, float eps, const int32_t* __restrict__ rows,
+                               const int32_t* __restrict__ d_R) {
+    __shared__ float scratch[33];
+    const int r = blockIdx.x;
+    int src = r;
+    if (rows) {
+        if (r >= *d_R) return;
+        src = rows[r];
+    }
+    const uint4* xin = reinterpret_cast<const uint4*>(x + (size_t)src * d);
+    const int nvec = d / 8;
+    constexpr int MAXV = 8;
+    uint4 buf[MAXV];
+    float ss = 0.f;
+#pragma unroll
+    for (int t = 0; t < MAXV; ++t) {
+        int i = threadIdx.x + t * blockDim.x;
+        if (i < nvec) {
+            buf[t] = xin[i];
+            const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&buf[t]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float2 f = __bfloat1622float2(b2[j]);
+                ss += f.x * f.x + f.y * f.y;
+            }
+        }
+    }
+    ss = block_sum(ss, scratch);
+    const float inv = rsqrtf(ss / (float)d + eps);
+    const uint4* g4 = reinterpret_cast<const uint4*>(gain);
+    uint4* o4 = reinterpret_cast<uint4*>(out + (size_t)r * d);
+#pragma unroll
+    for (int t = 0; t < MAXV; ++t) {
+        int i = threadIdx.x + t * blockDim.x;
+        if (i < nvec) {
+            uint4 gv = g4[i], ov;
+            const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&buf[t]);
+            const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gv);
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float2 f = __bfloat1622float2(b2[j]), g = __bfloat1622float2(g2[j]);
+                o2[j] = __floats2bfloat162_rn(f.x * inv * g.x, f.y * inv * g.y);
+            }
+            o4[i] = ov;
+        }
+    }
+}
+
+// Rotate-half RoPE in place on the Q and K heads of qkv [B*L, (nq + 2 nkv) * hd], and transpose V into
+// vt [B, nkv, hd, Lp] (keys contiguous) for the P.V product.  cs = [max_seq, hd/2] (cos, sin) table.
+// grid = (B*L, nq + 2*nkv), block = hd/2 threads.
+__global__ void rope_vt_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ vt,
+                               const float2* __restrict__ cs, int L, int Lp, int nq, int nkv, int hd) {
+    const int row = blockIdx.x, head = blockIdx.y, j = threadIdx.x, half = hd >> 1;
+    const int pos = row % L, b = row / L;
+    __nv_bfloat16* base = qkv + (size_t)row * (nq + 2 * nkv) * hd + (size_t)head * hd;
+    if (head < nq + nkv) {
+        const float2 c = cs[(size_t)pos * half + j];
+        const float x0 = __bfloat162float(base[j]), x1 = __bfloat162float(base[j + half]);
+        base[j] = __float2bfloat16_rn(x0 * c.x - x1 * c.y);
+        base[j + half] = __float2bfloat16_rn(x1 * c.x + x0 * c.y);
+    } else {
+        const int kvh = head - nq - nkv;
+        __nv_bfloat16* dst = vt + ((size_t)(b * nkv + kvh) * hd) * Lp + pos;
+        dst[(size_t)j * Lp] = base[j];
+        dst[(size_t)(j + half) * Lp] = base[j + half];
+    }
+}
+
+// Active rows of the step: every position of [lo_b, hi_b) that holds mask_id, in (b, i) order.
+// Single CTA.  rows[r] = b*L + i; *d_R = count.  With `state`, each sequence uses its own block.
+__global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restrict__ tokens, int B, int L,
+                                                          int32_t mask_id, int blk_lo, int blk_hi,
+                                                          const SeqState* __restrict__ state, int P, int block_len,
+                                                          int n_blocks, int32_t* __restrict__ rows,
+                                                          int32_t* __restrict__ d_R) {
+    __shared__ int warp_counts[32];
+    __shared__ int total;
+    const int tid = threadIdx.x, wid = tid >> 5, ln = tid & 31;
+    if (tid == 0) total = 0;
+    __syncthreads();
+    for (int b = 0; b < B; ++b) {
+        int lo = blk_lo, hi = blk_hi;
+        if (state) {
+            const int blk = state[b].blk;
+            if (blk >= n_blocks) continue;
+            lo = P + blk * block_len;
+            hi = lo + block_len;
+        }
+        for (int base = lo; base < hi; base += blockDim.x) {
+            const int i = base + tid;
+            const bool c = (i < hi) && tokens[(size_t)b * L + i] == mask_id;
+            const uint32_t bal = __ballot_sync(0xffffffffu, c);
+            if (ln == 0) warp_counts[wid] = __popc(bal);
+            __syncthreads();
+            int off = total;
+            for (int w = 0; w < wid; ++w) off += warp_counts[w];
+            if (c) rows[off + __popc(bal & ((1u << ln) - 1u))] = b * L + i;
+            __syncthreads();
+            if (tid == 0) {
+                int t = 0;
+                for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += warp_counts[w];
+                total += t;
+            }
+            __syncthreads();
+        }
+    }
+    if (tid == 0) *d_R = total;
+}
+
+// Merge the per-chunk partial statistics of each active row (chunks ascend through the vocabulary, so
+// "strictly greater" keeps the lowest index on ties) and scatter them to the [B, L] outputs.
+__global__ void merge_stats_kernel(const float4* __restrict__ partials, int R_pad, int grid_gemm, int n_vt,
+                                   const int32_t* __restrict__ rows, const int32_t* __restrict__ d_R,
+                                   float* __restrict__ top1, float* __restrict__ top2, float* __restrict__ sumexp,
+                                   int32_t* __restrict__ argmax) {
+    const int R = *d_R;
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    int n_rb = (R + 127) / 128;
+    int n_ch = grid_gemm / n_rb;
+    if (n_ch > n_vt) n_ch = n_vt;
+    float m1 = -INFINITY, m2 = -INFINITY, S = 0.f;
+    int i1 = 0x7fffffff;
+    for (int c = 0; c < n_ch; ++c) {
+        const float4 t = partials[(size_t)c * R_pad + r];
+        const float bm1 = t.x, bm2 = t.z, bS = t.w;
+        const int bi1 = __float_as_int(t.y);
+        const float nm = fmaxf(m1, bm1);
+        m2 = fmaxf(fmaxf(m2, bm2), fminf(m1, bm1));
+        S = S * expf(m1 - nm) + bS * expf(bm1 - nm);
+        if (bm1 > m1) i1 = bi1;
+        m1 = nm;
+    }
+    const int flat = rows[r];
+    top1[flat] = m1;
+    top2[flat] = m2;
+    sumexp[flat] = S;
+    argmax[flat] = i1;
+}
+
+// x = [prompt ; mask_id * G]  and fresh loop state  (Algorithm 1, initialisation)
+__global__ void init_canvas_kernel(const int32_t* __restrict__ prompt, int32_t* __restrict__ x, int B, int P, int G,
+                                   int32_t mask_id, SeqState* __restrict__ state) {
+    const int L = P + G;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < B * L) {
+        const int b = idx / L, i = idx % L;
+        x[idx] = (i < P) ? prompt[(size_t)b * P + i] : mask_id;
+    }
+    if (idx < B) state[idx] = SeqState{0, 0, 0, G > 0 ? 1 : 0};
+}
+
+}  // namespace jot

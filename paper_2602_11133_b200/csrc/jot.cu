@@ -1,0 +1,625 @@
+// C ABI of the JoT denoising-step library: argument checks, workspace layout, tensor maps, kernel
+// launches and the generate loop of Algorithm 1.  All arithmetic of the step lives in the kernels
+// (gemm.cuh, attention.cuh, glue.cuh, accept.cuh); nothing here computes on the host.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/jot.h"
+#include "accept.cuh"
+#include "attention.cuh"
+#include "gemm.cuh"
+#include "glue.cuh"
+
+using namespace jot;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<int64_t> g_launches{0};
+
+#define JOT_CUDA(expr)                                  \
+    do {                                                \
+        cudaError_t e_ = (expr);                        \
+        if (e_ != cudaSuccess) {                        \
+            g_last_cuda_error = (int)e_;                \
+            return JOT_ERR_CUDA;                        \
+        }                                               \
+    } while (0)
+#define JOT_TRY(expr)              \
+    do {                           \
+        int s_ = (expr);           \
+        if (s_ != JOT_OK) return s_; \
+    } while (0)
+
+inline int launch_check() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return JOT_ERR_CUDA;
+    }
+    return JOT_OK;
+}
+
+// ---------------------------------------------------------------- device facts
+struct DeviceInfo {
+    int ok = 0, sms = 0, status = JOT_OK;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+};
+
+int device_info(DeviceInfo** out) {
+    static thread_local DeviceInfo cache[64];
+    int dev = 0;
+    JOT_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return JOT_ERR_DEVICE;
+    DeviceInfo& di = cache[dev];
+    if (!di.ok) {
+        int major = 0;
+        JOT_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        JOT_CUDA(cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev));
+        if (major != 10) return JOT_ERR_DEVICE;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        JOT_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return JOT_ERR_DEVICE;
+        di.encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+        di.ok = 1;
+    }
+    *out = &di;
+    return JOT_OK;
+}
+
+// bf16 row-major [rows, cols] (row stride ld elements), boxes of 64 columns x box_rows rows, 128-byte swizzle;
+// out-of-range elements read as zero.
+int make_map_2d(const DeviceInfo* di, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld,
+                uint32_t box_rows) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = di->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = (int)cudaErrorInvalidValue;
+        return JOT_ERR_CUDA;
+    }
+    return JOT_OK;
+}
+// qkv viewed as (column, position, sequence)
+int make_map_qkv(const DeviceInfo* di, CUtensorMap* map, const void* ptr, uint64_t B, uint64_t L, uint64_t cols) {
+    cuuint64_t dims[3] = {cols, L, B};
+    cuuint64_t strides[2] = {cols * 2, L * cols * 2};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = di->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = (int)cudaErrorInvalidValue;
+        return JOT_ERR_CUDA;
+    }
+    return JOT_OK;
+}
+
+// ---------------------------------------------------------------- GEMM launch
+template <int BN, int EPI>
+int launch_gemm_t(const GemmParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int grid, cudaStream_t st) {
+    static thread_local bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev & 63]) {
+        JOT_CUDA(cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      GemmSmem<BN>::DYN_BYTES));
+        attr_set[dev & 63] = true;
+    }
+    gemm_kernel<BN, EPI><<<grid, kGemmThreads, GemmSmem<BN>::DYN_BYTES, st>>>(p, tmA, tmB);
+    return launch_check();
+}
+
+// Tile width for a plain projection: the one that needs the least (waves x tile width).
+int pick_bn(int M, int n_out, int sms) {
+    long m_blks = (M + 127) / 128;
+    long t256 = m_blks * ((n_out + 255) / 256), t128 = m_blks * ((n_out + 127) / 128);
+    long c256 = ((t256 + sms - 1) / sms) * 256, c128 = ((t128 + sms - 1) / sms) * 128;
+    return c128 < c256 ? 128 : 256;
+}
+
+struct WeightMaps {     // one weight matrix as B operand, for both tile widths
+    CUtensorMap m128, m256;
+};
+
+int make_weight_maps(const DeviceInfo* di, WeightMaps* w, const void* ptr, int rows, int cols, bool swiglu) {
+    // swiglu tiles fetch gate and up rows as two boxes of half the tile width
+    JOT_TRY(make_map_2d(di, &w->m128, ptr, rows, cols, cols, swiglu ? 64 : 128));
+    JOT_TRY(make_map_2d(di, &w->m256, ptr, rows, cols, cols, swiglu ? 128 : 256));
+    return JOT_OK;
+}
+
+int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, int epi, GemmParams p, cudaStream_t st) {
+    const int n_out = (epi == EPI_SWIGLU) ? p.N / 2 : p.N;
+    int bn = pick_bn(p.M, epi == EPI_SWIGLU ? 2 * n_out : n_out, di->sms);
+    const int bn_out = (epi == EPI_SWIGLU) ? bn / 2 : bn;
+    long tiles = (long)((p.M + 127) / 128) * ((n_out + bn_out - 1) / bn_out);
+    int grid = (int)(tiles < di->sms ? tiles : di->sms);
+    if (grid <= 0) return JOT_OK;
+    if (epi == EPI_STORE)
+        return bn == 256 ? launch_gemm_t<256, EPI_STORE>(p, tmA, w.m256, grid, st)
+                         : launch_gemm_t<128, EPI_STORE>(p, tmA, w.m128, grid, st);
+    return bn == 256 ? launch_gemm_t<256, EPI_SWIGLU>(p, tmA, w.m256, grid, st)
+                     : launch_gemm_t<128, EPI_SWIGLU>(p, tmA, w.m128, grid, st);
+}
+
+template <int HD>
+int launch_attention_t(const AttnParams& p, const CUtensorMap& tq, const CUtensorMap& tv, dim3 grid, cudaStream_t st) {
+    static thread_local bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev & 63]) {
+        JOT_CUDA(cudaFuncSetAttribute(attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      AttnSmem<HD>::DYN_BYTES));
+        attr_set[dev & 63] = true;
+    }
+    attention_kernel<HD><<<grid, kAttnThreads, AttnSmem<HD>::DYN_BYTES, st>>>(p, tq, tv);
+    return launch_check();
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+// ---------------------------------------------------------------- model object
+struct jot_model {
+    jot_model_config cfg;
+    int max_batch, max_seq;
+    DeviceInfo* di;
+    // borrowed weights
+    const __nv_bfloat16 *embed, *lm_head, *final_norm;
+    std::vector<const __nv_bfloat16*> attn_norm, mlp_norm;
+    std::vector<WeightMaps> wqkv, wo, wgu, wdown;
+    WeightMaps wlm;
+    // workspace slices
+    int32_t* ctrl;        // [0] status, [1] R, [2] n_unfinished
+    float2* rope_cs;
+    __nv_bfloat16 *h, *a, *qkv, *vt, *attn, *act, *hsel;
+    int32_t* rows;
+    float4* partials;
+    int R_cap;
+    int32_t* canvas;      // generate: tokens [max_batch * max_seq]
+    float *g_top1, *g_top2, *g_sumexp;
+    int32_t* g_argmax;
+    SeqState* state;
+    AcceptParamsDev* params_dev;
+    // activation tensor maps, re-encoded when (B, L) changes
+    int map_B = -1, map_L = -1;
+    CUtensorMap tm_a, tm_attn, tm_act, tm_hsel, tm_qkv3, tm_vt;
+    int32_t* h_pinned = nullptr;    // pinned host words for loop control read-back
+};
+
+namespace {
+
+struct Layout {
+    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, partials, canvas, top1, top2, sumexp, argmax, state, params,
+        total;
+};
+
+bool config_ok(const jot_model_config* c) {
+    if (!c) return false;
+    if (c->n_layers < 0 || c->d_model <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->d_ff <= 0 || c->vocab <= 1)
+        return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->d_model % 64 || c->d_ff % 64 || c->vocab % 8 || c->n_q_heads % c->n_kv_heads) return false;
+    if (c->d_model > 16384) return false;
+    if (c->mask_id < 0 || c->mask_id >= c->vocab) return false;
+    return true;
+}
+
+Layout make_layout(const jot_model_config* c, int max_batch, int max_seq) {
+    Layout l;
+    const size_t M = (size_t)max_batch * max_seq, R_cap = align_up(M, 128);
+    const size_t qkv_cols = (size_t)(c->n_q_heads + 2 * c->n_kv_heads) * c->head_dim;
+    const size_t Lp = align_up((size_t)max_seq, 8);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes, 1024);
+        return o;
+    };
+    l.ctrl = take(1024);
+    l.rope = take((size_t)max_seq * (c->head_dim / 2) * sizeof(float2));
+    l.h = take(M * c->d_model * 2);
+    l.a = take(M * c->d_model * 2);
+    l.qkv = take(M * qkv_cols * 2);
+    l.vt = take((size_t)max_batch * c->n_kv_heads * c->head_dim * Lp * 2);
+    l.attn = take(M * (size_t)c->n_q_heads * c->head_dim * 2);
+    l.act = take(M * (size_t)c->d_ff * 2);
+    l.hsel = take(R_cap * c->d_model * 2);
+    l.rows = take(R_cap * 4);
+    l.partials = take((size_t)256 * R_cap * sizeof(float4));   // up to 256 vocabulary chunks
+    l.canvas = take(M * 4);
+    l.top1 = take(M * 4);
+    l.top2 = take(M * 4);
+    l.sumexp = take(M * 4);
+    l.argmax = take(M * 4);
+    l.state = take((size_t)max_batch * sizeof(SeqState));
+    l.params = take((size_t)max_batch * sizeof(AcceptParamsDev));
+    l.total = off;
+    return l;
+}
+
+int encode_activation_maps(jot_model* m, int B, int L) {
+    if (m->map_B == B && m->map_L == L) return JOT_OK;
+    const jot_model_config& c = m->cfg;
+    const int M = B * L;
+    const int qkv_cols = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+    const int Lp = (int)align_up((size_t)L, 8);
+    JOT_TRY(make_map_2d(m->di, &m->tm_a, m->a, M, c.d_model, c.d_model, 128));
+    JOT_TRY(make_map_2d(m->di, &m->tm_attn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim, 128));
+    JOT_TRY(make_map_2d(m->di, &m->tm_act, m->act, M, c.d_ff, c.d_ff, 128));
+    JOT_TRY(make_map_2d(m->di, &m->tm_hsel, m->hsel, m->R_cap, c.d_model, c.d_model, 128));
+    JOT_TRY(make_map_qkv(m->di, &m->tm_qkv3, m->qkv, B, L, qkv_cols));
+    JOT_TRY(make_map_2d(m->di, &m->tm_vt, m->vt, (uint64_t)B * c.n_kv_heads * c.head_dim, L, Lp, c.head_dim));
+    m->map_B = B;
+    m->map_L = L;
+    return JOT_OK;
+}
+
+// Transformer body: tokens [B, L] -> residual stream m->h [B*L, d] (before the final norm).
+int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream_t st) {
+    const jot_model_config& c = m->cfg;
+    const int M = B * L, d = c.d_model, hd = c.head_dim, nq = c.n_q_heads, nkv = c.n_kv_heads;
+    const int qkv_cols = (nq + 2 * nkv) * hd;
+    const int Lp = (int)align_up((size_t)L, 8);
+    JOT_TRY(encode_activation_maps(m, B, L));
+    int32_t* status = m->ctrl;
+
+    embed_kernel<<<M, 128, 0, st>>>(d_tokens, m->embed, m->h, d);
+    JOT_TRY(launch_check());
+    for (int l = 0; l < c.n_layers; ++l) {
+        rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->attn_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+        JOT_TRY(launch_check());
+        GemmParams p{};
+        p.M = M; p.N = qkv_cols; p.K = d; p.C = m->qkv; p.ldc = qkv_cols; p.status = status;
+        JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_STORE, p, st));
+        rope_vt_kernel<<<dim3(M, nq + 2 * nkv), hd / 2, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv, hd);
+        JOT_TRY(launch_check());
+        AttnParams ap{};
+        ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
+        ap.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
+        dim3 grid((L + 127) / 128, nq, B);
+        if (hd == 128) JOT_TRY(launch_attention_t<128>(ap, m->tm_qkv3, m->tm_vt, grid, st));
+        else JOT_TRY(launch_attention_t<64>(ap, m->tm_qkv3, m->tm_vt, grid, st));
+        p = GemmParams{};
+        p.M = M; p.N = d; p.K = nq * hd; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
+        JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st));
+        rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->mlp_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+        JOT_TRY(launch_check());
+        p = GemmParams{};
+        p.M = M; p.N = 2 * c.d_ff; p.K = d; p.C = m->act; p.ldc = c.d_ff; p.status = status;
+        JOT_TRY(run_gemm(m->di, m->tm_a, m->wgu[l], EPI_SWIGLU, p, st));
+        p = GemmParams{};
+        p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
+        JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st));
+    }
+    return JOT_OK;
+}
+
+// hsel (active rows, already gathered) -> merged statistics scattered to the [B, L] outputs
+int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, const float* bump_val, float* top1,
+                      float* top2, float* sumexp, int32_t* argmax, int M, cudaStream_t st) {
+    const jot_model_config& c = m->cfg;
+    GemmParams p{};
+    p.M = m->R_cap; p.N = c.vocab; p.K = c.d_model; p.status = m->ctrl;
+    p.d_R = m->ctrl + 1; p.rows = m->rows; p.bump_id = bump_id; p.bump_val = bump_val;
+    p.mask_col = exclude_mask ? c.mask_id : -1;
+    p.partials = m->partials; p.R_pad = m->R_cap;
+    const int grid = m->di->sms > 256 ? 256 : m->di->sms;
+    // few active rows: the head streams W once and is bandwidth bound -> narrower tiles balance the SMs better
+    const int bn = (M <= 256) ? 128 : 256;
+    if (bn == 256) JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
+    else JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+    const int n_vt = (c.vocab + bn - 1) / bn;
+    merge_stats_kernel<<<(m->R_cap + 127) / 128, 128, 0, st>>>(m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
+                                                               top1, top2, sumexp, argmax);
+    return launch_check();
+}
+
+// copy rows of a [*, d] bf16 matrix selected by `rows` (only r < *d_R)
+__global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int d,
+                                   const int32_t* __restrict__ rows, const int32_t* __restrict__ d_R) {
+    const int r = blockIdx.x;
+    if (r >= *d_R) return;
+    const uint4* s = reinterpret_cast<const uint4*>(src + (size_t)rows[r] * d);
+    uint4* t = reinterpret_cast<uint4*>(dst + (size_t)r * d);
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
+}
+
+int check_step_args(const jot_model* m, const void* tokens, int B, int L, int blk_lo, int blk_hi, const void* bump_id,
+                    const void* bump_val, const void* o1, const void* o2, const void* o3, const void* o4) {
+    if (!m || !tokens || !o1 || !o2 || !o3 || !o4) return JOT_ERR_ARG;
+    if ((bump_id == nullptr) != (bump_val == nullptr)) return JOT_ERR_ARG;
+    if (B <= 0 || L <= 0 || blk_lo < 0 || blk_hi > L || blk_lo > blk_hi) return JOT_ERR_ARG;
+    if (B > m->max_batch || L > m->max_seq) return JOT_ERR_SHAPE;
+    return JOT_OK;
+}
+
+int read_status(jot_model* m, cudaStream_t st) {
+    JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 4, cudaMemcpyDeviceToHost, st));
+    JOT_CUDA(cudaStreamSynchronize(st));
+    return m->h_pinned[0] ? JOT_ERR_TIMEOUT : JOT_OK;
+}
+
+int launch_accept(const AcceptArgs& a, cudaStream_t st) {
+    const size_t smem = accept_smem_bytes(a.L);
+    if (smem > 200 * 1024) return JOT_ERR_SHAPE;
+    if (smem > 48 * 1024) {
+        JOT_CUDA(cudaFuncSetAttribute(accept_freeze_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    accept_freeze_kernel<<<a.B, kAcceptThreads, smem, st>>>(a);
+    return launch_check();
+}
+
+bool params_ok(const jot_params* p) { return p && p->D >= 1 && p->D <= kMaxD; }
+
+}  // namespace
+
+// ---------------------------------------------------------------- exported functions
+extern "C" {
+
+const char* jot_status_string(int s) {
+    switch (s) {
+        case JOT_OK: return "ok";
+        case JOT_ERR_ARG: return "invalid argument";
+        case JOT_ERR_SHAPE: return "unsupported shape";
+        case JOT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case JOT_ERR_CUDA: return "CUDA call failed";
+        case JOT_ERR_TIMEOUT: return "bounded device wait expired";
+        case JOT_ERR_DEVICE: return "device or driver not supported (needs sm_100 and tensor-map support)";
+        default: return "unknown status";
+    }
+}
+
+int jot_last_cuda_error(void) { return g_last_cuda_error; }
+int64_t jot_launch_count(void) { return g_launches.load(); }
+
+size_t jot_workspace_bytes(const jot_model_config* cfg, int max_batch, int max_seq) {
+    if (!config_ok(cfg) || max_batch <= 0 || max_seq <= 0) return 0;
+    return make_layout(cfg, max_batch, max_seq).total;
+}
+
+int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_batch, int max_seq, void* ws,
+                   size_t ws_bytes, jot_model** out) {
+    if (!cfg || !w || !out) return JOT_ERR_ARG;
+    *out = nullptr;
+    if (max_batch <= 0 || max_seq <= 0) return JOT_ERR_ARG;
+    if (!config_ok(cfg)) return JOT_ERR_SHAPE;
+    if (!w->embed || !w->lm_head || !w->final_norm) return JOT_ERR_ARG;
+    if (cfg->n_layers > 0 && (!w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm || !w->w_gate_up || !w->w_down))
+        return JOT_ERR_ARG;
+    const Layout lay = make_layout(cfg, max_batch, max_seq);
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 1023) || ws_bytes < lay.total) return JOT_ERR_WORKSPACE;
+    DeviceInfo* di = nullptr;
+    JOT_TRY(device_info(&di));
+
+    jot_model* m = new (std::nothrow) jot_model();
+    if (!m) return JOT_ERR_ARG;
+    m->cfg = *cfg;
+    m->max_batch = max_batch;
+    m->max_seq = max_seq;
+    m->di = di;
+    m->embed = (const __nv_bfloat16*)w->embed;
+    m->lm_head = (const __nv_bfloat16*)w->lm_head;
+    m->final_norm = (const __nv_bfloat16*)w->final_norm;
+    uint8_t* base = (uint8_t*)ws;
+    m->ctrl = (int32_t*)(base + lay.ctrl);
+    m->rope_cs = (float2*)(base + lay.rope);
+    m->h = (__nv_bfloat16*)(base + lay.h);
+    m->a = (__nv_bfloat16*)(base + lay.a);
+    m->qkv = (__nv_bfloat16*)(base + lay.qkv);
+    m->vt = (__nv_bfloat16*)(base + lay.vt);
+    m->attn = (__nv_bfloat16*)(base + lay.attn);
+    m->act = (__nv_bfloat16*)(base + lay.act);
+    m->hsel = (__nv_bfloat16*)(base + lay.hsel);
+    m->rows = (int32_t*)(base + lay.rows);
+    m->partials = (float4*)(base + lay.partials);
+    m->R_cap = (int)align_up((size_t)max_batch * max_seq, 128);
+    m->canvas = (int32_t*)(base + lay.canvas);
+    m->g_top1 = (float*)(base + lay.top1);
+    m->g_top2 = (float*)(base + lay.top2);
+    m->g_sumexp = (float*)(base + lay.sumexp);
+    m->g_argmax = (int32_t*)(base + lay.argmax);
+    m->state = (SeqState*)(base + lay.state);
+    m->params_dev = (AcceptParamsDev*)(base + lay.params);
+
+    int rc = JOT_OK;
+    auto fail = [&](int code) {
+        if (m->h_pinned) cudaFreeHost(m->h_pinned);
+        delete m;
+        return code;
+    };
+    const int d = cfg->d_model, hd = cfg->head_dim, nq = cfg->n_q_heads, nkv = cfg->n_kv_heads;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->mlp_norm[l] || !w->w_gate_up[l] || !w->w_down[l])
+            return fail(JOT_ERR_ARG);
+        m->attn_norm.push_back((const __nv_bfloat16*)w->attn_norm[l]);
+        m->mlp_norm.push_back((const __nv_bfloat16*)w->mlp_norm[l]);
+        WeightMaps wm;
+        if ((rc = make_weight_maps(di, &wm, w->wqkv[l], (nq + 2 * nkv) * hd, d, false)) != JOT_OK) return fail(rc);
+        m->wqkv.push_back(wm);
+        if ((rc = make_weight_maps(di, &wm, w->wo[l], d, nq * hd, false)) != JOT_OK) return fail(rc);
+        m->wo.push_back(wm);
+        if ((rc = make_weight_maps(di, &wm, w->w_gate_up[l], 2 * cfg->d_ff, d, true)) != JOT_OK) return fail(rc);
+        m->wgu.push_back(wm);
+        if ((rc = make_weight_maps(di, &wm, w->w_down[l], d, cfg->d_ff, false)) != JOT_OK) return fail(rc);
+        m->wdown.push_back(wm);
+    }
+    if ((rc = make_weight_maps(di, &m->wlm, w->lm_head, cfg->vocab, d, false)) != JOT_OK) return fail(rc);
+
+    // tables: cos/sin of pos * theta^(-2j/hd), evaluated in double on the host once
+    std::vector<float2> cs((size_t)max_seq * (hd / 2));
+    for (int pos = 0; pos < max_seq; ++pos)
+        for (int j = 0; j < hd / 2; ++j) {
+            const double ang = (double)pos * std::pow((double)cfg->rope_theta, -2.0 * j / hd);
+            cs[(size_t)pos * (hd / 2) + j] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+        }
+    cudaError_t e = cudaMemcpy(m->rope_cs, cs.data(), cs.size() * sizeof(float2), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(m->ctrl, 0, 1024);
+    if (e == cudaSuccess) e = cudaMemset(m->hsel, 0, (size_t)m->R_cap * d * 2);
+    if (e == cudaSuccess) e = cudaMemset(m->rows, 0, (size_t)m->R_cap * 4);
+    if (e == cudaSuccess) e = cudaHostAlloc((void**)&m->h_pinned, 64 + (size_t)max_batch * sizeof(SeqState), cudaHostAllocDefault);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return fail(JOT_ERR_CUDA);
+    }
+    *out = m;
+    return JOT_OK;
+}
+
+int jot_free_model(jot_model* m) {
+    if (!m) return JOT_ERR_ARG;
+    if (m->h_pinned) cudaFreeHost(m->h_pinned);
+    delete m;
+    return JOT_OK;
+}
+
+int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi,
+                      int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val, float* d_top1,
+                      float* d_top2, float* d_sumexp, int32_t* d_argmax, void* stream) {
+    JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
+    if (!d_hidden) return JOT_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    JOT_TRY(encode_activation_maps(m, B, L));
+    build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+                                          m->ctrl + 1);
+    JOT_TRY(launch_check());
+    gather_rows_kernel<<<B * L, 128, 0, st>>>((const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
+                                              m->ctrl + 1);
+    JOT_TRY(launch_check());
+    JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
+                              B * (blk_hi - blk_lo), st));
+    return read_status(m, st);
+}
+
+int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi, int exclude_mask_token,
+                     const int32_t* d_bump_id, const float* d_bump_val, float* d_top1, float* d_top2, float* d_sumexp,
+                     int32_t* d_argmax, void* stream) {
+    JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
+    cudaStream_t st = (cudaStream_t)stream;
+    JOT_TRY(forward_body(m, d_tokens, B, L, st));
+    build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+                                          m->ctrl + 1);
+    JOT_TRY(launch_check());
+    rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
+                                          m->ctrl + 1);
+    JOT_TRY(launch_check());
+    JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
+                              B * (blk_hi - blk_lo), st));
+    return read_status(m, st);
+}
+
+int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask_id, int32_t* d_tokens, int B, int L,
+                      int blk_lo, int blk_hi, int k_transfer, const float* d_top1, const float* d_top2,
+                      const float* d_sumexp, const int32_t* d_argmax, int32_t* d_n_masked, uint8_t* d_exit_reason,
+                      int16_t* d_exit_step, int step_index, void* stream) {
+    if (!params || !d_tokens || !d_top1 || !d_top2 || !d_sumexp || !d_argmax) return JOT_ERR_ARG;
+    if (B <= 0 || L <= 0 || blk_lo < 0 || blk_hi > L || blk_lo > blk_hi || k_transfer < 0) return JOT_ERR_ARG;
+    if (per_seq_params) return JOT_ERR_ARG;   // per-sequence parameters are available through jot_generate
+    if (!params_ok(params)) return JOT_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    AcceptArgs a{};
+    a.uniform = AcceptParamsDev{params->tau_max, params->tau_min, params->gamma, params->D, params->eps,
+                                params->schedule_after_exit};
+    a.params = nullptr;
+    a.mask_id = mask_id; a.tokens = d_tokens; a.B = B; a.L = L;
+    a.blk_lo = blk_lo; a.blk_hi = blk_hi; a.k_transfer = k_transfer;
+    a.top1 = d_top1; a.top2 = d_top2; a.sumexp = d_sumexp; a.argmax = d_argmax;
+    a.n_masked = d_n_masked; a.exit_reason = d_exit_reason; a.exit_step = d_exit_step; a.step_index = step_index;
+    a.state = nullptr;
+    JOT_TRY(launch_accept(a, st));
+    return JOT_OK;
+}
+
+int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, const jot_gen_config* gen,
+                 const int32_t* d_prompt, int B, int P, const int32_t* d_bump_id, const float* d_bump_val,
+                 int32_t* d_out_tokens, int32_t* h_steps_used, int32_t* h_forward_passes, void* stream) {
+    if (!m || !params || !gen || !d_out_tokens || !h_steps_used) return JOT_ERR_ARG;
+    if ((d_bump_id == nullptr) != (d_bump_val == nullptr)) return JOT_ERR_ARG;
+    if (B <= 0 || P < 0 || gen->gen_len <= 0 || gen->steps <= 0 || gen->block_len <= 0) return JOT_ERR_ARG;
+    if (P > 0 && !d_prompt) return JOT_ERR_ARG;
+    if (gen->gen_len % gen->block_len) return JOT_ERR_ARG;
+    const int nb = gen->gen_len / gen->block_len;
+    if (gen->steps % nb) return JOT_ERR_ARG;
+    const int Tb = gen->steps / nb, L = P + gen->gen_len;
+    if (B > m->max_batch || L > m->max_seq) return JOT_ERR_SHAPE;
+    const int n_par = per_seq_params ? B : 1;
+    for (int i = 0; i < n_par; ++i)
+        if (!params_ok(params + i)) return JOT_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    static_assert(sizeof(AcceptParamsDev) == sizeof(jot_params), "parameter struct layouts must agree");
+    JOT_CUDA(cudaMemcpyAsync(m->params_dev, params, (size_t)n_par * sizeof(jot_params), cudaMemcpyHostToDevice, st));
+    init_canvas_kernel<<<(B * L + 255) / 256, 256, 0, st>>>(d_prompt, m->canvas, B, P, gen->gen_len, m->cfg.mask_id,
+                                                           m->state);
+    JOT_TRY(launch_check());
+    int passes = 0;
+    for (int it = 0; it < gen->steps; ++it) {
+        JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
+        JOT_TRY(forward_body(m, m->canvas, B, L, st));
+        build_rows_kernel<<<1, 1024, 0, st>>>(m->canvas, B, L, m->cfg.mask_id, 0, 0, m->state, P, gen->block_len, nb,
+                                              m->rows, m->ctrl + 1);
+        JOT_TRY(launch_check());
+        rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
+                                              m->ctrl + 1);
+        JOT_TRY(launch_check());
+        JOT_TRY(lm_head_from_hsel(m, gen->exclude_mask_token, d_bump_id, d_bump_val, m->g_top1, m->g_top2, m->g_sumexp,
+                                  m->g_argmax, B * gen->block_len, st));
+        AcceptArgs a{};
+        a.params = m->params_dev; a.per_seq_params = per_seq_params ? 1 : 0;
+        a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
+        a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp; a.argmax = m->g_argmax;
+        a.step_index = it + 1;
+        a.state = m->state; a.P = P; a.block_len = gen->block_len; a.n_blocks = nb; a.steps_per_block = Tb;
+        a.n_unfinished = m->ctrl + 2;
+        JOT_TRY(launch_accept(a, st));
+        ++passes;
+        JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 12, cudaMemcpyDeviceToHost, st));
+        JOT_CUDA(cudaStreamSynchronize(st));
+        if (m->h_pinned[0]) return JOT_ERR_TIMEOUT;
+        if (m->h_pinned[2] == 0) break;
+    }
+    JOT_CUDA(cudaMemcpyAsync(d_out_tokens, m->canvas, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
+    SeqState* hs = reinterpret_cast<SeqState*>(m->h_pinned + 16);
+    JOT_CUDA(cudaMemcpyAsync(hs, m->state, (size_t)B * sizeof(SeqState), cudaMemcpyDeviceToHost, st));
+    JOT_CUDA(cudaStreamSynchronize(st));
+    for (int b = 0; b < B; ++b) h_steps_used[b] = hs[b].steps_used;
+    if (h_forward_passes) *h_forward_passes = passes;
+    return JOT_OK;
+}
+
+int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
+                  int32_t* d_status, void* stream) {
+    if (!d_A || !d_W || !d_C) return JOT_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return JOT_ERR_ARG;
+    if (N % 8 || K % 8) return JOT_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_A) | reinterpret_cast<uintptr_t>(d_W) | reinterpret_cast<uintptr_t>(d_C) |
+         reinterpret_cast<uintptr_t>(d_residual)) & 15)
+        return JOT_ERR_ARG;
+    DeviceInfo* di = nullptr;
+    JOT_TRY(device_info(&di));
+    CUtensorMap tmA;
+    WeightMaps wm;
+    JOT_TRY(make_map_2d(di, &tmA, d_A, M, K, K, 128));
+    JOT_TRY(make_weight_maps(di, &wm, d_W, N, K, false));
+    GemmParams p{};
+    p.M = M; p.N = N; p.K = K; p.C = (__nv_bfloat16*)d_C; p.residual = (const __nv_bfloat16*)d_residual; p.ldc = N;
+    p.status = d_status;
+    return run_gemm(di, tmA, wm, EPI_STORE, p, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,249 @@
+"""ctypes binding of libjot.so: argument marshalling only.
+
+Every step of the JoT denoising path runs inside the CUDA library; this module turns torch tensors
+into raw device pointers, checks dtypes/shapes, and raises on any non-zero status.  There is no
+fallback: if the library is missing or fails to load, importing the binding's functions raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import dataclasses
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libjot.so")
+
+EXPORTS = [
+    "jot_status_string", "jot_last_cuda_error", "jot_workspace_bytes", "jot_init_model", "jot_free_model",
+    "jot_denoise_step", "jot_lm_head_stats", "jot_accept_freeze", "jot_generate", "jot_gemm_bf16",
+    "jot_launch_count",
+]
+
+
+class JotError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib().jot_status_string(status).decode()
+        cuda = _lib().jot_last_cuda_error()
+        super().__init__(f"{where}: {msg} (status {status}, cuda error {cuda})")
+
+
+class Params(C.Structure):
+    """tau_max, tau_min, gamma, D of Algorithm 1; eps of Eq. 4."""
+    _fields_ = [("tau_max", C.c_float), ("tau_min", C.c_float), ("gamma", C.c_float), ("D", C.c_int32),
+                ("eps", C.c_float), ("schedule_after_exit", C.c_int32)]
+
+    def __init__(self, tau_max=90.0, tau_min=1.0, gamma=0.5, D=8, eps=1e-12, schedule_after_exit=0):
+        super().__init__(tau_max, tau_min, gamma, D, eps, schedule_after_exit)
+
+
+class ModelConfig(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32), ("mask_id", C.c_int32),
+                ("rope_theta", C.c_float), ("rms_eps", C.c_float)]
+
+
+class _Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("attn_norm", C.POINTER(C.c_void_p)), ("wqkv", C.POINTER(C.c_void_p)), ("wo", C.POINTER(C.c_void_p)),
+                ("mlp_norm", C.POINTER(C.c_void_p)), ("w_gate_up", C.POINTER(C.c_void_p)),
+                ("w_down", C.POINTER(C.c_void_p))]
+
+
+class GenConfig(C.Structure):
+    _fields_ = [("gen_len", C.c_int32), ("steps", C.c_int32), ("block_len", C.c_int32),
+                ("exclude_mask_token", C.c_int32)]
+
+
+_LIB = None
+
+
+def _lib():
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_11133_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        lib = C.CDLL(LIB_PATH)
+        lib.jot_status_string.restype = C.c_char_p
+        lib.jot_status_string.argtypes = [C.c_int]
+        lib.jot_last_cuda_error.restype = C.c_int
+        lib.jot_workspace_bytes.restype = C.c_size_t
+        lib.jot_workspace_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int, C.c_int]
+        lib.jot_init_model.argtypes = [C.POINTER(ModelConfig), C.POINTER(_Weights), C.c_int, C.c_int, C.c_void_p,
+                                       C.c_size_t, C.POINTER(C.c_void_p)]
+        lib.jot_free_model.argtypes = [C.c_void_p]
+        step_args = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                     C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.jot_denoise_step.argtypes = [C.c_void_p, C.c_void_p] + step_args
+        lib.jot_lm_head_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + step_args
+        lib.jot_accept_freeze.argtypes = [C.POINTER(Params), C.c_int, C.c_int32, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                          C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+        lib.jot_generate.argtypes = [C.c_void_p, C.POINTER(Params), C.c_int, C.POINTER(GenConfig), C.c_void_p, C.c_int,
+                                     C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32),
+                                     C.POINTER(C.c_int32), C.c_void_p]
+        lib.jot_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                      C.c_void_p, C.c_void_p]
+        lib.jot_launch_count.restype = C.c_int64
+        _LIB = lib
+    return _LIB
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise JotError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def launch_count() -> int:
+    return int(_lib().jot_launch_count())
+
+
+@dataclasses.dataclass
+class Stats:
+    """Per-position softmax statistics, each [B, L]; only active rows are written."""
+    top1: torch.Tensor
+    top2: torch.Tensor
+    sumexp: torch.Tensor
+    argmax: torch.Tensor
+
+    @staticmethod
+    def empty(B: int, L: int, device) -> "Stats":
+        return Stats(torch.zeros(B, L, dtype=torch.float32, device=device),
+                     torch.zeros(B, L, dtype=torch.float32, device=device),
+                     torch.ones(B, L, dtype=torch.float32, device=device),
+                     torch.zeros(B, L, dtype=torch.int32, device=device))
+
+
+class Model:
+    """Owner of the device workspace and the library's model handle.  Weights are borrowed."""
+
+    def __init__(self, geometry, weights: dict, max_batch: int, max_seq: int):
+        g = geometry
+        self.geometry = g
+        self.cfg = ModelConfig(len(weights["layers"]), g.d_model, g.n_q_heads, g.n_kv_heads, g.head_dim, g.d_ff,
+                               g.vocab, g.mask_id, g.rope_theta, g.rms_eps)
+        self.weights = weights           # keep the tensors alive
+        self.max_batch, self.max_seq = max_batch, max_seq
+        lib = _lib()
+        nbytes = lib.jot_workspace_bytes(C.byref(self.cfg), max_batch, max_seq)
+        if nbytes == 0:
+            raise JotError(-2, "jot_workspace_bytes")
+        dev = weights["lm_head"].device
+        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        base = (self.workspace.data_ptr() + 1023) // 1024 * 1024
+        nl = self.cfg.n_layers
+        arr = lambda key: (C.c_void_p * max(nl, 1))(*[_ptr(lw[key], torch.bfloat16, key) for lw in weights["layers"]])
+        self._arrays = [arr(k) for k in ("attn_norm", "wqkv", "wo", "mlp_norm", "w_gate_up", "w_down")]
+        w = _Weights(_ptr(weights["embed"], torch.bfloat16, "embed"), _ptr(weights["lm_head"], torch.bfloat16, "lm_head"),
+                     _ptr(weights["final_norm"], torch.bfloat16, "final_norm"),
+                     *[C.cast(a, C.POINTER(C.c_void_p)) for a in self._arrays])
+        handle = C.c_void_p()
+        _check(lib.jot_init_model(C.byref(self.cfg), C.byref(w), max_batch, max_seq, base, nbytes, C.byref(handle)),
+               "jot_init_model")
+        self.handle = handle
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib().jot_free_model(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- one step -------------------------------------------------------------------------------
+    def denoise_step(self, tokens: torch.Tensor, blk_lo: int, blk_hi: int, out: Optional[Stats] = None,
+                     exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
+                     bump_val: Optional[torch.Tensor] = None) -> Stats:
+        B, L = tokens.shape
+        out = out or Stats.empty(B, L, tokens.device)
+        _check(_lib().jot_denoise_step(self.handle, _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo, blk_hi,
+                                       int(exclude_mask_token), _ptr(bump_id, torch.int32, "bump_id"),
+                                       _ptr(bump_val, torch.float32, "bump_val"), out.top1.data_ptr(),
+                                       out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), _stream()),
+               "jot_denoise_step")
+        return out
+
+    def lm_head_stats(self, hidden: torch.Tensor, tokens: torch.Tensor, blk_lo: int, blk_hi: int,
+                      out: Optional[Stats] = None, exclude_mask_token: bool = True,
+                      bump_id: Optional[torch.Tensor] = None, bump_val: Optional[torch.Tensor] = None) -> Stats:
+        B, L = tokens.shape
+        if hidden.shape != (B * L, self.cfg.d_model):
+            raise ValueError("hidden must be [B*L, d_model]")
+        out = out or Stats.empty(B, L, tokens.device)
+        _check(_lib().jot_lm_head_stats(self.handle, _ptr(hidden, torch.bfloat16, "hidden"),
+                                        _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo, blk_hi,
+                                        int(exclude_mask_token), _ptr(bump_id, torch.int32, "bump_id"),
+                                        _ptr(bump_val, torch.float32, "bump_val"), out.top1.data_ptr(),
+                                        out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), _stream()),
+               "jot_lm_head_stats")
+        return out
+
+    # ---- Algorithm 1 ----------------------------------------------------------------------------
+    def generate(self, prompt: torch.Tensor, gen_len: int, steps: int, params, block_len: Optional[int] = None,
+                 exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
+                 bump_val: Optional[torch.Tensor] = None):
+        """Returns (tokens [B, P+gen_len] int32 on device, steps_used list[int], forward_passes int)."""
+        B, P = prompt.shape
+        per_seq = isinstance(params, (list, tuple))
+        if per_seq:
+            if len(params) != B:
+                raise ValueError("need one Params per sequence")
+            parr = (Params * B)(*params)
+        else:
+            parr = (Params * 1)(params)
+        gen = GenConfig(gen_len, steps, block_len or gen_len, int(exclude_mask_token))
+        out = torch.empty(B, P + gen_len, dtype=torch.int32, device=prompt.device)
+        used = (C.c_int32 * B)()
+        passes = C.c_int32(0)
+        _check(_lib().jot_generate(self.handle, parr, int(per_seq), C.byref(gen), _ptr(prompt, torch.int32, "prompt"), B,
+                                   P, _ptr(bump_id, torch.int32, "bump_id"), _ptr(bump_val, torch.float32, "bump_val"),
+                                   out.data_ptr(), used, C.byref(passes), _stream()), "jot_generate")
+        return out, list(used), int(passes.value)
+
+
+def accept_freeze(params: Params, mask_id: int, tokens: torch.Tensor, blk_lo: int, blk_hi: int, k_transfer: int,
+                  stats: Stats, n_masked: Optional[torch.Tensor] = None, exit_reason: Optional[torch.Tensor] = None,
+                  exit_step: Optional[torch.Tensor] = None, step_index: int = 0) -> None:
+    """In-place acceptance / freeze update of tokens [B, L] (Section 4.1, Algorithm 1)."""
+    B, L = tokens.shape
+    _check(_lib().jot_accept_freeze(C.byref(params), 0, mask_id, _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo,
+                                    blk_hi, k_transfer, _ptr(stats.top1, torch.float32, "top1"),
+                                    _ptr(stats.top2, torch.float32, "top2"), _ptr(stats.sumexp, torch.float32, "sumexp"),
+                                    _ptr(stats.argmax, torch.int32, "argmax"), _ptr(n_masked, torch.int32, "n_masked"),
+                                    _ptr(exit_reason, torch.uint8, "exit_reason"),
+                                    _ptr(exit_step, torch.int16, "exit_step"), step_index, _stream()),
+           "jot_accept_freeze")
+
+
+def gemm_bf16(a: torch.Tensor, w: torch.Tensor, residual: Optional[torch.Tensor] = None,
+              out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """out[M, N] = a[M, K] @ w[N, K]^T (+ residual), bf16 in/out, fp32 accumulate."""
+    M, K = a.shape
+    N = w.shape[0]
+    out = torch.empty(M, N, dtype=torch.bfloat16, device=a.device) if out is None else out
+    status = torch.zeros(1, dtype=torch.int32, device=a.device)
+    _check(_lib().jot_gemm_bf16(_ptr(a, torch.bfloat16, "a"), _ptr(w, torch.bfloat16, "w"),
+                                _ptr(residual, torch.bfloat16, "residual"), _ptr(out, torch.bfloat16, "out"), M, N, K,
+                                status.data_ptr(), _stream()), "jot_gemm_bf16")
+    if int(status.item()) != 0:
+        raise JotError(-5, "jot_gemm_bf16")
+    return out

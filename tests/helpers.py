@@ -1,0 +1,67 @@
+"""Shared helpers for the GPU parity tests: oracle-side glue and comparison rules.
+
+Tolerances (bf16 path): logits-derived values within 2e-2 relative to the row's logit scale; argmax and
+accept/freeze decisions bit-exact except where the oracle itself says the decision is within 1e-3 of
+flipping (top-2 logit gap < 1e-3, or |r - tau| <= 1e-3 tau); those positions are counted and reported.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Tuple
+
+import numpy as np
+import torch
+
+from oracle import jot_oracle as jo
+from oracle import model_oracle as mo
+
+REL_TOL = 2e-2
+GAP_TOL = 1e-3
+
+
+def oracle_stats_for_rows(logits_rows: torch.Tensor, mask_id) -> List[jo.RowStats]:
+    return [jo.row_stats(logits_rows[r].numpy(), mask_id) for r in range(logits_rows.shape[0])]
+
+
+def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowStats], rel=REL_TOL):
+    """Returns (n_checked, n_near_tie).  Raises AssertionError on a real mismatch."""
+    near = 0
+    for r, st in enumerate(want):
+        scale = max(abs(st.m1), abs(st.m2), 1.0)
+        assert abs(got_top1[r] - st.m1) <= rel * scale, (r, got_top1[r], st.m1)
+        assert abs(got_top2[r] - st.m2) <= rel * scale, (r, got_top2[r], st.m2)
+        # log-sum-exp agrees to the logit tolerance  <=> S agrees to a relative factor
+        assert abs(math.log(got_sumexp[r]) - math.log(st.S)) <= rel * scale, (r, got_sumexp[r], st.S)
+        if st.m1 - st.m2 < GAP_TOL:
+            near += 1                     # top-2 gap below 1e-3: either index is a valid argmax
+        else:
+            assert int(got_argmax[r]) == st.i1, (r, int(got_argmax[r]), st.i1, st.m1 - st.m2)
+    return len(want), near
+
+
+def stats_dict_from_arrays(top1, top2, sumexp, argmax, b: int, positions) -> Dict[int, jo.RowStats]:
+    return {i: jo.RowStats(float(top1[b, i]), int(argmax[b, i]), float(top2[b, i]), float(sumexp[b, i]))
+            for i in positions}
+
+
+def oracle_accept_batch(tokens: torch.Tensor, top1, top2, sumexp, argmax, params: jo.JotParams, mask_id: int,
+                        lo: int, hi: int, k: int, schedule_after_exit=False) -> Tuple[torch.Tensor, List[jo.StepReport]]:
+    """Run the oracle's accept/freeze on every sequence, statistics given as [B, L] float/int arrays."""
+    out = tokens.clone()
+    reps = []
+    for b in range(tokens.shape[0]):
+        x = tokens[b].tolist()
+        A = [i for i in range(lo, hi) if x[i] == mask_id]
+        st = stats_dict_from_arrays(top1, top2, sumexp, argmax, b, A)
+        rep = jo.accept_freeze(x, st, params, mask_id, lo, hi, k, schedule_after_exit)
+        out[b] = torch.tensor(x, dtype=tokens.dtype)
+        reps.append(rep)
+    return out, reps
+
+
+def bf16_matmul_oracle(a: torch.Tensor, w: torch.Tensor, residual=None) -> torch.Tensor:
+    """float64 a @ w^T (+ residual), the definition the projection kernel is checked against."""
+    out = a.double() @ w.double().T
+    if residual is not None:
+        out = out + residual.double()
+    return out

@@ -1,0 +1,215 @@
+"""GPU parity tests of the individual kernels against the CPU oracle, through the C ABI."""
+import math
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import (GAP_TOL, bf16_matmul_oracle, compare_stats, oracle_accept_batch, oracle_stats_for_rows)
+from oracle import jot_oracle as jo
+from oracle import model_oracle as mo
+from paper_2602_11133_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def jot():
+    from paper_2602_11133_b200 import jot as binding
+    binding._lib()          # fail loudly if the library is missing
+    return binding
+
+
+# ---------------------------------------------------------------- projection GEMM
+@pytest.mark.parametrize("M,N,K", [
+    (128, 256, 64), (96, 768, 256), (96, 256, 704), (384, 4096, 4096), (200, 1408, 256),
+    (384, 12288, 4096), (1000, 3584, 1024), (130, 136, 72),
+])
+@pytest.mark.parametrize("with_res", [False, True])
+def test_gemm_matches_float64_definition(jot, M, N, K, with_res):
+    a = inputs.normal(1, "a", (M, K), 1.0).cuda()
+    w = inputs.normal(1, "w", (N, K), 0.05).cuda()
+    res = inputs.normal(1, "r", (M, N), 1.0).cuda() if with_res else None
+    out = jot.gemm_bf16(a, w, res)
+    torch.cuda.synchronize()
+    want = bf16_matmul_oracle(a.cpu(), w.cpu(), None if res is None else res.cpu())
+    got = out.cpu().double()
+    # one bf16 rounding of an fp32-accumulated value: half an ulp (2^-9 relative) plus accumulation noise
+    err = (got - want).abs()
+    tol = 2.0 ** -8 * want.abs() + 1e-3 * want.abs().max()
+    assert (err <= tol).all(), f"max err {err.max().item()} at {torch.nonzero(err > tol)[:4].tolist()}"
+    # and it is not trivially zero
+    assert got.abs().max().item() > 0.1
+
+
+def test_gemm_residual_in_place(jot):
+    a = inputs.normal(2, "a", (384, 512), 1.0).cuda()
+    w = inputs.normal(2, "w", (1024, 512), 0.05).cuda()
+    h = inputs.normal(2, "h", (384, 1024), 1.0).cuda()
+    want = bf16_matmul_oracle(a.cpu(), w.cpu(), h.cpu())
+    jot.gemm_bf16(a, w, h, out=h)
+    torch.cuda.synchronize()
+    err = (h.cpu().double() - want).abs()
+    assert (err <= 2.0 ** -8 * want.abs() + 1e-3 * want.abs().max()).all()
+
+
+# ---------------------------------------------------------------- acceptance / freeze
+def random_accept_case(seed, B, L, P, mask_id, V, hot=0.3):
+    rng = np.random.default_rng(seed)
+    tokens = rng.integers(0, V - 1, size=(B, L)).astype(np.int32)
+    tokens[tokens >= mask_id] += 1
+    masked = rng.random((B, L)) < 0.55
+    masked[:, :P] = False
+    tokens[masked] = mask_id
+    gap = rng.random((B, L)) * np.where(rng.random((B, L)) < hot, 9.0, 0.6)
+    top1 = (rng.standard_normal((B, L)) * 2 + 4).astype(np.float32)
+    top2 = (top1 - gap).astype(np.float32)
+    sumexp = (1.0 + np.exp(top2.astype(np.float64) - top1) + rng.random((B, L)) * 5).astype(np.float32)
+    argmax = rng.integers(0, V - 1, size=(B, L)).astype(np.int32)
+    argmax[argmax >= mask_id] += 1
+    return tokens, top1, top2, sumexp, argmax
+
+
+@pytest.mark.parametrize("B,L,P,lo,hi,k", [
+    (1, 96, 32, 32, 96, 1), (8, 384, 128, 128, 384, 1), (3, 704, 192, 224, 256, 1), (4, 100, 0, 0, 100, 3),
+    (2, 1000, 10, 10, 1000, 7), (16, 704, 192, 192, 704, 2), (2, 33, 5, 5, 33, 40),
+])
+@pytest.mark.parametrize("params", [jo.DREAM_DEFAULT, jo.LLADA_DEFAULT, jo.JotParams(60, 1, 0.7, 8),
+                                    jo.JotParams(90, 30, 0.9, 16), jo.JotParams(120, 1, 0.3, 32)])
+def test_accept_freeze_matches_oracle(jot, B, L, P, lo, hi, k, params):
+    V, mask_id = 5000, 4321
+    tokens, top1, top2, sumexp, argmax = random_accept_case(B * 1000 + L, B, L, P, mask_id, V)
+    want, reps = oracle_accept_batch(torch.from_numpy(tokens), top1, top2, sumexp, argmax, params, mask_id, lo, hi, k)
+    d_tok = torch.from_numpy(tokens).cuda()
+    st = jot.Stats(torch.from_numpy(top1).cuda(), torch.from_numpy(top2).cuda(), torch.from_numpy(sumexp).cuda(),
+                   torch.from_numpy(argmax).cuda())
+    n_masked = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    reason = torch.zeros(B, L, dtype=torch.uint8, device="cuda")
+    estep = torch.zeros(B, L, dtype=torch.int16, device="cuda")
+    jot.accept_freeze(jot.Params(params.tau_max, params.tau_min, params.gamma, params.D, params.eps), mask_id, d_tok,
+                      lo, hi, k, st, n_masked, reason, estep, step_index=7)
+    torch.cuda.synchronize()
+    got = d_tok.cpu()
+    near = 0
+    for b in range(B):
+        nm = set(reps[b].near_margin)
+        near += len(nm)
+        for i in range(L):
+            if i in nm:
+                # the early-exit decision may legitimately differ; either outcome must be a valid one
+                assert int(got[b, i]) in (mask_id, int(argmax[b, i]))
+                continue
+            assert int(got[b, i]) == int(want[b, i]), (b, i, reps[b].ratio.get(i), reps[b].tau.get(i))
+        if not nm:
+            assert int(n_masked[b]) == int((want[b, lo:hi] == mask_id).sum())
+            exp_reason = np.zeros(L, dtype=np.uint8)
+            for i in reps[b].exited:
+                exp_reason[i] |= 1
+            for i in reps[b].scheduled:
+                exp_reason[i] |= 2
+            assert np.array_equal(reason[b].cpu().numpy(), exp_reason)
+            assert np.array_equal(estep[b].cpu().numpy(), np.where(exp_reason > 0, 7, 0).astype(np.int16))
+    assert near <= max(2, B * L // 200)
+    # untouched outside the block, prompt never changes, frozen tokens never change
+    assert torch.equal(got[:, :lo], torch.from_numpy(tokens)[:, :lo])
+    assert torch.equal(got[:, hi:], torch.from_numpy(tokens)[:, hi:])
+    keep = torch.from_numpy(tokens) != mask_id
+    assert torch.equal(got[keep], torch.from_numpy(tokens)[keep])
+
+
+def test_accept_freeze_degenerate_cases(jot):
+    V, mask_id, B, L = 100, 99, 2, 64
+    tokens, top1, top2, sumexp, argmax = random_accept_case(5, B, L, 8, mask_id, V)
+    st = jot.Stats(*[torch.from_numpy(t).cuda() for t in (top1, top2, sumexp, argmax)])
+    # nothing masked in the block: no change, zero left
+    t0 = torch.from_numpy(tokens).cuda()
+    t0[:, 8:16] = 5
+    before = t0.clone()
+    n = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    jot.accept_freeze(jot.Params(), mask_id, t0, 8, 16, 1, st, n)
+    assert torch.equal(t0, before) and n.tolist() == [0, 0]
+    # empty range
+    jot.accept_freeze(jot.Params(), mask_id, t0, 20, 20, 1, st, n)
+    assert torch.equal(t0, before) and n.tolist() == [0, 0]
+    # threshold 0: everything in the block is finalised at once (uncapped), k = 0
+    t1 = torch.from_numpy(tokens).cuda()
+    jot.accept_freeze(jot.Params(0.0, 0.0, 0.5, 8), mask_id, t1, 8, L, 0, st, n)
+    assert (t1[:, 8:] != mask_id).all() and n.tolist() == [0, 0]
+    # threshold +inf and k = 0: nothing happens
+    t2 = torch.from_numpy(tokens).cuda()
+    jot.accept_freeze(jot.Params(float("inf"), float("inf"), 0.5, 8), mask_id, t2, 8, L, 0, st, n)
+    assert torch.equal(t2.cpu(), torch.from_numpy(tokens))
+    # invalid arguments are refused on the host
+    with pytest.raises(jot.JotError):
+        jot.accept_freeze(jot.Params(D=0), mask_id, t2, 8, L, 1, st, n)
+    with pytest.raises(jot.JotError):
+        jot.accept_freeze(jot.Params(D=33), mask_id, t2, 8, L, 1, st, n)
+    with pytest.raises(jot.JotError):
+        jot.accept_freeze(jot.Params(), mask_id, t2, 8, L + 1, 1, st, n)
+
+
+# ---------------------------------------------------------------- fused LM head + statistics
+def lm_head_model(jot, d, V, mask_id, w_lm, max_batch, max_seq):
+    g = inputs.ModelGeometry(0, d, 1, 1, 64, 64, V, mask_id)
+    weights = {"embed": w_lm, "lm_head": w_lm, "final_norm": torch.ones(d, dtype=torch.bfloat16, device="cuda"),
+               "layers": []}
+    return jot.Model(g, weights, max_batch, max_seq)
+
+
+@pytest.mark.parametrize("B,P,G,d,V,bump", [
+    (1, 32, 64, 256, 4096, False),        # tiny model's head
+    (2, 40, 200, 512, 5000, True),        # ragged vocabulary tail (5000 = 19.5 tiles of 256), 2 row blocks
+    (3, 100, 284, 256, 1032, True),       # several row blocks, vocabulary smaller than the grid
+    (8, 128, 256, 1024, 12800, True),     # > 1024 active rows: wide-tile path
+])
+def test_lm_head_stats_match_oracle(jot, B, P, G, d, V, bump):
+    mask_id = V - 7
+    case = inputs.lm_head_case(3, B, P, G, d, V, mask_id, device="cuda")
+    model = lm_head_model(jot, d, V, mask_id, case.w, B, P + G)
+    L = P + G
+    st = model.lm_head_stats(case.hidden, case.tokens, P, L, exclude_mask_token=True,
+                             bump_id=case.bump_id if bump else None, bump_val=case.bump_val if bump else None)
+    torch.cuda.synchronize()
+    tok = case.tokens.cpu()
+    rows = [(b, i) for b in range(B) for i in range(P, L) if int(tok[b, i]) == mask_id]
+    assert len(rows) > 0
+    flat = torch.tensor([b * L + i for b, i in rows])
+    logits = mo.lm_head_logits(case.hidden.cpu()[flat], case.w.cpu(),
+                               case.bump_id.cpu().view(-1)[flat] if bump else None,
+                               case.bump_val.cpu().view(-1)[flat] if bump else None)
+    want = oracle_stats_for_rows(logits, mask_id)
+    pick = lambda t: t.cpu().view(-1)[flat].numpy()
+    n, near = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), want, rel=1e-3)
+    assert near <= max(1, n // 100)
+    # rows that are not active are left untouched
+    untouched = torch.ones(B * L, dtype=torch.bool)
+    untouched[flat] = False
+    assert (st.sumexp.cpu().view(-1)[untouched] == 1.0).all() and (st.argmax.cpu().view(-1)[untouched] == 0).all()
+    model.close()
+
+
+def test_lm_head_mask_token_and_ties(jot):
+    # hidden = one-hot rows and a crafted head make exact ties and a dominant mask column
+    d, V, mask_id, B, L = 64, 512, 100, 1, 128
+    w = torch.zeros(V, d, dtype=torch.bfloat16)
+    w[100, 0] = 8.0          # mask column would win
+    w[7, 0] = 2.0
+    w[300, 0] = 2.0          # exact tie with column 7 -> argmax 7, top2 == top1
+    w[450, 0] = 1.0
+    hidden = torch.zeros(B * L, d, dtype=torch.bfloat16)
+    hidden[:, 0] = 1.0
+    tokens = torch.full((B, L), mask_id, dtype=torch.int32)
+    model = lm_head_model(jot, d, V, mask_id, w.cuda(), B, L)
+    st = model.lm_head_stats(hidden.cuda(), tokens.cuda(), 0, L, exclude_mask_token=True)
+    assert (st.argmax.cpu() == 7).all() and (st.top1.cpu() == 2.0).all() and (st.top2.cpu() == 2.0).all()
+    S = 2.0 + math.exp(-1.0) + (V - 4) * math.exp(-2.0)
+    assert torch.allclose(st.sumexp.cpu(), torch.full((B, L), S), rtol=1e-5)
+    st = model.lm_head_stats(hidden.cuda(), tokens.cuda(), 0, L, exclude_mask_token=False)
+    assert (st.argmax.cpu() == 100).all() and (st.top1.cpu() == 8.0).all() and (st.top2.cpu() == 2.0).all()
+    # no active rows at all: a no-op
+    tokens[:] = 3
+    out = jot.Stats.empty(B, L, "cuda")
+    model.lm_head_stats(hidden.cuda(), tokens.cuda(), 0, L, out=out)
+    assert (out.sumexp == 1.0).all()
+    model.close()
