@@ -164,6 +164,19 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
 int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
                   int32_t* d_status, void* stream);
 
+/* Optional timing of the kernels a model launches, by class, with CUDA events recorded on the launching
+ * stream around each launch.  jot_profile(m, 1) starts (and clears) the accumulation, jot_profile(m, 0)
+ * stops it; jot_profile_read waits for the recorded events and returns, per class, the accumulated
+ * device milliseconds and the number of timed spans (host arrays of at least JOT_PROF_CLASSES entries).
+ * Classes time single kernels except ROWS (active-row list + final norm / gather, two kernels). */
+enum {
+    JOT_PROF_EMBED = 0, JOT_PROF_RMSNORM, JOT_PROF_GEMM_QKV, JOT_PROF_ROPE, JOT_PROF_ATTENTION, JOT_PROF_GEMM_O,
+    JOT_PROF_GEMM_GATE_UP, JOT_PROF_GEMM_DOWN, JOT_PROF_ROWS, JOT_PROF_LM_HEAD, JOT_PROF_MERGE, JOT_PROF_ACCEPT,
+    JOT_PROF_CLASSES
+};
+int jot_profile(jot_model* m, int enable);
+int jot_profile_read(jot_model* m, double* ms, int64_t* launches, int n_classes);
+
 /* Number of kernels this library has launched from the calling process so far. */
 int64_t jot_launch_count(void);
 

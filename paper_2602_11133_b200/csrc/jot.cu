@@ -201,9 +201,45 @@ struct jot_model {
     int map_B = -1, map_L = -1;
     CUtensorMap tm_a, tm_attn, tm_act, tm_hsel, tm_qkv3, tm_vt;
     int32_t* h_pinned = nullptr;    // pinned host words for loop control read-back
+    // optional per-kernel-class timing with CUDA events on the launching stream
+    bool profiling = false;
+    std::vector<cudaEvent_t> ev_pool;
+    size_t ev_used = 0;
+    struct Span { int cls; cudaEvent_t a, b; };
+    std::vector<Span> spans;
+    double prof_ms[JOT_PROF_CLASSES] = {};
+    int64_t prof_n[JOT_PROF_CLASSES] = {};
 };
 
 namespace {
+
+// Brackets one kernel launch with a pair of events while profiling is on.
+struct ProfScope {
+    jot_model* m;
+    cudaStream_t st;
+    cudaEvent_t b = nullptr;
+    int cls;
+    ProfScope(jot_model* m_, int cls_, cudaStream_t st_) : m(m_), st(st_), cls(cls_) {
+        if (!m->profiling) return;
+        cudaEvent_t a = next();
+        b = next();
+        if (a && b) {
+            cudaEventRecord(a, st);
+            m->spans.push_back({cls, a, b});
+        }
+    }
+    ~ProfScope() {
+        if (b) cudaEventRecord(b, st);
+    }
+    cudaEvent_t next() {
+        if (m->ev_used == m->ev_pool.size()) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+            m->ev_pool.push_back(e);
+        }
+        return m->ev_pool[m->ev_used++];
+    }
+};
 
 struct Layout {
     size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, partials, canvas, top1, top2, sumexp, argmax, state, params,
@@ -280,33 +316,60 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
     JOT_TRY(encode_activation_maps(m, B, L));
     int32_t* status = m->ctrl;
 
-    embed_kernel<<<M, 128, 0, st>>>(d_tokens, m->embed, m->h, d);
+    {
+        ProfScope ps(m, JOT_PROF_EMBED, st);
+        embed_kernel<<<M, 128, 0, st>>>(d_tokens, m->embed, m->h, d);
+    }
     JOT_TRY(launch_check());
     for (int l = 0; l < c.n_layers; ++l) {
-        rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->attn_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+        {
+            ProfScope ps(m, JOT_PROF_RMSNORM, st);
+            rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->attn_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+        }
         JOT_TRY(launch_check());
         GemmParams p{};
         p.M = M; p.N = qkv_cols; p.K = d; p.C = m->qkv; p.ldc = qkv_cols; p.status = status;
-        JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_STORE, p, st));
-        rope_vt_kernel<<<dim3(M, nq + 2 * nkv), hd / 2, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv, hd);
+        {
+            ProfScope ps(m, JOT_PROF_GEMM_QKV, st);
+            JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_STORE, p, st));
+        }
+        {
+            ProfScope ps(m, JOT_PROF_ROPE, st);
+            rope_vt_kernel<<<dim3(M, nq + 2 * nkv), hd / 2, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv, hd);
+        }
         JOT_TRY(launch_check());
         AttnParams ap{};
         ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
         ap.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
         dim3 grid((L + 127) / 128, nq, B);
-        if (hd == 128) JOT_TRY(launch_attention_t<128>(ap, m->tm_qkv3, m->tm_vt, grid, st));
-        else JOT_TRY(launch_attention_t<64>(ap, m->tm_qkv3, m->tm_vt, grid, st));
+        {
+            ProfScope ps(m, JOT_PROF_ATTENTION, st);
+            if (hd == 128) JOT_TRY(launch_attention_t<128>(ap, m->tm_qkv3, m->tm_vt, grid, st));
+            else JOT_TRY(launch_attention_t<64>(ap, m->tm_qkv3, m->tm_vt, grid, st));
+        }
         p = GemmParams{};
         p.M = M; p.N = d; p.K = nq * hd; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
-        JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st));
-        rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->mlp_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+        {
+            ProfScope ps(m, JOT_PROF_GEMM_O, st);
+            JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st));
+        }
+        {
+            ProfScope ps(m, JOT_PROF_RMSNORM, st);
+            rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->mlp_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+        }
         JOT_TRY(launch_check());
         p = GemmParams{};
         p.M = M; p.N = 2 * c.d_ff; p.K = d; p.C = m->act; p.ldc = c.d_ff; p.status = status;
-        JOT_TRY(run_gemm(m->di, m->tm_a, m->wgu[l], EPI_SWIGLU, p, st));
+        {
+            ProfScope ps(m, JOT_PROF_GEMM_GATE_UP, st);
+            JOT_TRY(run_gemm(m->di, m->tm_a, m->wgu[l], EPI_SWIGLU, p, st));
+        }
         p = GemmParams{};
         p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
-        JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st));
+        {
+            ProfScope ps(m, JOT_PROF_GEMM_DOWN, st);
+            JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st));
+        }
     }
     return JOT_OK;
 }
@@ -323,9 +386,13 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     const int grid = m->di->sms > 256 ? 256 : m->di->sms;
     // few active rows: the head streams W once and is bandwidth bound -> narrower tiles balance the SMs better
     const int bn = (M <= 256) ? 128 : 256;
-    if (bn == 256) JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
-    else JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+    {
+        ProfScope ps(m, JOT_PROF_LM_HEAD, st);
+        if (bn == 256) JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
+        else JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+    }
     const int n_vt = (c.vocab + bn - 1) / bn;
+    ProfScope ps(m, JOT_PROF_MERGE, st);
     merge_stats_kernel<<<(m->R_cap + 127) / 128, 128, 0, st>>>(m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
                                                                top1, top2, sumexp, argmax);
     return launch_check();
@@ -485,6 +552,7 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
 int jot_free_model(jot_model* m) {
     if (!m) return JOT_ERR_ARG;
     if (m->h_pinned) cudaFreeHost(m->h_pinned);
+    for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
     delete m;
     return JOT_OK;
 }
@@ -496,12 +564,15 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
     if (!d_hidden) return JOT_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     JOT_TRY(encode_activation_maps(m, B, L));
-    build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
-                                          m->ctrl + 1);
-    JOT_TRY(launch_check());
-    gather_rows_kernel<<<B * L, 128, 0, st>>>((const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
+    {
+        ProfScope ps(m, JOT_PROF_ROWS, st);
+        build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
                                               m->ctrl + 1);
-    JOT_TRY(launch_check());
+        JOT_TRY(launch_check());
+        gather_rows_kernel<<<B * L, 128, 0, st>>>((const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
+                                                  m->ctrl + 1);
+        JOT_TRY(launch_check());
+    }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
                               B * (blk_hi - blk_lo), st));
     return read_status(m, st);
@@ -513,12 +584,15 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
     JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
     cudaStream_t st = (cudaStream_t)stream;
     JOT_TRY(forward_body(m, d_tokens, B, L, st));
-    build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
-                                          m->ctrl + 1);
-    JOT_TRY(launch_check());
-    rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
-                                          m->ctrl + 1);
-    JOT_TRY(launch_check());
+    {
+        ProfScope ps(m, JOT_PROF_ROWS, st);
+        build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+                                              m->ctrl + 1);
+        JOT_TRY(launch_check());
+        rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
+                                              m->ctrl + 1);
+        JOT_TRY(launch_check());
+    }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
                               B * (blk_hi - blk_lo), st));
     return read_status(m, st);
@@ -571,12 +645,15 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     for (int it = 0; it < gen->steps; ++it) {
         JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
         JOT_TRY(forward_body(m, m->canvas, B, L, st));
-        build_rows_kernel<<<1, 1024, 0, st>>>(m->canvas, B, L, m->cfg.mask_id, 0, 0, m->state, P, gen->block_len, nb,
-                                              m->rows, m->ctrl + 1);
-        JOT_TRY(launch_check());
-        rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
-                                              m->ctrl + 1);
-        JOT_TRY(launch_check());
+        {
+            ProfScope ps(m, JOT_PROF_ROWS, st);
+            build_rows_kernel<<<1, 1024, 0, st>>>(m->canvas, B, L, m->cfg.mask_id, 0, 0, m->state, P, gen->block_len,
+                                                  nb, m->rows, m->ctrl + 1);
+            JOT_TRY(launch_check());
+            rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps,
+                                                  m->rows, m->ctrl + 1);
+            JOT_TRY(launch_check());
+        }
         JOT_TRY(lm_head_from_hsel(m, gen->exclude_mask_token, d_bump_id, d_bump_val, m->g_top1, m->g_top2, m->g_sumexp,
                                   m->g_argmax, B * gen->block_len, st));
         AcceptArgs a{};
@@ -586,7 +663,10 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         a.step_index = it + 1;
         a.state = m->state; a.P = P; a.block_len = gen->block_len; a.n_blocks = nb; a.steps_per_block = Tb;
         a.n_unfinished = m->ctrl + 2;
-        JOT_TRY(launch_accept(a, st));
+        {
+            ProfScope ps(m, JOT_PROF_ACCEPT, st);
+            JOT_TRY(launch_accept(a, st));
+        }
         ++passes;
         JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 12, cudaMemcpyDeviceToHost, st));
         JOT_CUDA(cudaStreamSynchronize(st));
@@ -599,6 +679,30 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     JOT_CUDA(cudaStreamSynchronize(st));
     for (int b = 0; b < B; ++b) h_steps_used[b] = hs[b].steps_used;
     if (h_forward_passes) *h_forward_passes = passes;
+    return JOT_OK;
+}
+
+int jot_profile(jot_model* m, int enable) {
+    if (!m) return JOT_ERR_ARG;
+    m->profiling = enable != 0;
+    m->spans.clear();
+    m->ev_used = 0;
+    for (int i = 0; i < JOT_PROF_CLASSES; ++i) { m->prof_ms[i] = 0; m->prof_n[i] = 0; }
+    return JOT_OK;
+}
+
+int jot_profile_read(jot_model* m, double* ms, int64_t* launches, int n_classes) {
+    if (!m || !ms || !launches || n_classes < JOT_PROF_CLASSES) return JOT_ERR_ARG;
+    for (const auto& sp : m->spans) {
+        JOT_CUDA(cudaEventSynchronize(sp.b));
+        float t = 0.f;
+        JOT_CUDA(cudaEventElapsedTime(&t, sp.a, sp.b));
+        m->prof_ms[sp.cls] += t;
+        m->prof_n[sp.cls] += 1;
+    }
+    m->spans.clear();
+    m->ev_used = 0;
+    for (int i = 0; i < JOT_PROF_CLASSES; ++i) { ms[i] = m->prof_ms[i]; launches[i] = m->prof_n[i]; }
     return JOT_OK;
 }
 

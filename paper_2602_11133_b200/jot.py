@@ -19,8 +19,11 @@ LIB_PATH = os.path.join(_HERE, "libjot.so")
 EXPORTS = [
     "jot_status_string", "jot_last_cuda_error", "jot_workspace_bytes", "jot_init_model", "jot_free_model",
     "jot_denoise_step", "jot_lm_head_stats", "jot_accept_freeze", "jot_generate", "jot_gemm_bf16",
-    "jot_launch_count",
+    "jot_launch_count", "jot_profile", "jot_profile_read",
 ]
+
+PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "rows",
+                "lm_head", "merge", "accept"]
 
 
 class JotError(RuntimeError):
@@ -89,6 +92,8 @@ def _lib():
         lib.jot_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                       C.c_void_p, C.c_void_p]
         lib.jot_launch_count.restype = C.c_int64
+        lib.jot_profile.argtypes = [C.c_void_p, C.c_int]
+        lib.jot_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int]
         _LIB = lib
     return _LIB
 
@@ -168,6 +173,17 @@ class Model:
             self.close()
         except Exception:
             pass
+
+    def profile(self, enable: bool) -> None:
+        """Start (and clear) or stop per-kernel-class event timing."""
+        _check(_lib().jot_profile(self.handle, int(enable)), "jot_profile")
+
+    def profile_read(self) -> dict:
+        """{class: (milliseconds, spans)} accumulated since profile(True)."""
+        n = len(PROF_CLASSES)
+        ms, cnt = (C.c_double * n)(), (C.c_int64 * n)()
+        _check(_lib().jot_profile_read(self.handle, ms, cnt, n), "jot_profile_read")
+        return {name: (ms[i], int(cnt[i])) for i, name in enumerate(PROF_CLASSES)}
 
     # ---- one step -------------------------------------------------------------------------------
     def denoise_step(self, tokens: torch.Tensor, blk_lo: int, blk_hi: int, out: Optional[Stats] = None,
