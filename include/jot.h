@@ -160,9 +160,12 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
 /* C[M, N] (bf16) = A[M, K] (bf16) . W[N, K]^T (bf16) with fp32 accumulation on the tensor cores,
  * optionally + residual[M, N] (bf16, may alias C).  The projection every layer of the forward is made
  * of, exported for testing and benchmarking.  K and N multiples of 8; pointers 16-byte aligned.
+ * d_scratch (device, optional, 16-byte aligned, scratch_bytes long): fp32 space for split-K partial
+ * sums, used when the output has too few tiles to fill the GPU and up to 4 * M * N * 4 bytes fit;
+ * NULL keeps K in one piece.
  * d_status: device int32 the kernel sets non-zero if a bounded wait expires (may be NULL). */
 int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
-                  int32_t* d_status, void* stream);
+                  void* d_scratch, size_t scratch_bytes, int32_t* d_status, void* stream);
 
 /* Optional timing of the kernels a model launches, by class, with CUDA events recorded on the launching
  * stream around each launch.  jot_profile(m, 1) starts (and clears) the accumulation, jot_profile(m, 0)

@@ -9,12 +9,14 @@
 //        EPI_SWIGLU  bf16(silu(gate) * up), gate/up from the two halves of W -> C[M, N/2]
 //        EPI_STATS   online (max, argmax, runner-up, sum-exp) per row over a range of vocabulary tiles;
 //                    the logits are never written (LM head of the denoising step)
+//        EPI_PARTIAL fp32 partial sums of one K range (split-K for projections with too few output
+//                    tiles to fill the SMs); splitk_reduce_kernel adds the ranges and the residual
 #pragma once
 #include "ptx.cuh"
 
 namespace jot {
 
-enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2 };
+enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2, EPI_PARTIAL = 3 };
 
 constexpr int kBM = 128;          // rows per tile = TMEM lanes
 constexpr int kBK = 64;           // bf16 elements per 128-byte swizzled smem row
@@ -26,6 +28,8 @@ struct GemmParams {
     const __nv_bfloat16* residual;  // EPI_STORE, nullable, same shape as C
     int ldc;                      // row stride of C and residual, elements
     int32_t* status;              // set non-zero when a bounded wait expired (nullable)
+    int split_k;                  // EPI_PARTIAL: number of K ranges (>= 1); otherwise ignored
+    float* partial;               // EPI_PARTIAL: [split_k][M][N] fp32
     // EPI_STATS only
     const int32_t* d_R;           // number of active rows (device)
     const int32_t* rows;          // [R] flat canvas index b*L+i of each active row
@@ -78,7 +82,8 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
     const int n_out = (EPI == EPI_SWIGLU) ? p.N / 2 : p.N;
     const int num_n = (n_out + BN_OUT - 1) / BN_OUT;
-    int total_tiles = num_m * num_n;
+    const int split = (EPI == EPI_PARTIAL) ? p.split_k : 1;
+    int total_tiles = num_m * num_n * split;
     int chunk = 0;
     if (EPI == EPI_STATS) {
         int R = *p.d_R, n_rb, n_ch;
@@ -93,6 +98,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         }
         total_tiles = n_count;
     }
+    int kb0 = 0, kb1 = num_kb, ks = 0;            // K-block range of the current work item
     auto tile_at = [&](int it, int& m_blk, int& n_blk) -> bool {
         if (EPI == EPI_STATS) {
             if (it >= total_tiles) return false;
@@ -102,6 +108,12 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         }
         int t = blockIdx.x + it * gridDim.x;
         if (t >= total_tiles) return false;
+        if (EPI == EPI_PARTIAL) {
+            ks = t % split;
+            t /= split;
+            kb0 = (int)((long long)ks * num_kb / split);
+            kb1 = (int)((long long)(ks + 1) * num_kb / split);
+        }
         m_blk = t % num_m;                        // row blocks fastest: neighbours share the W tile
         n_blk = t / num_m;
         return true;
@@ -141,7 +153,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
             int m_blk, n_blk;
             bool ok = true;
             for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
                     uint8_t* sA = smem + stage * SM::STAGE_BYTES;
                     uint8_t* sB = sA + SM::A_BYTES;
@@ -170,7 +182,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
                 if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abortp)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + stage * SM::STAGE_BYTES);
@@ -178,7 +190,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k) {
                         umma_bf16(d_tmem, umma_desc_k128(a_addr + k * 32), umma_desc_k128(b_addr + k * 32), IDESC,
-                                  (kb | k) != 0);
+                                  (kb > kb0) || (k != 0));
                     }
                     umma_commit(&empty_bar[stage]);       // smem stage reusable once these MMAs retire
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -253,6 +265,22 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
                                 *reinterpret_cast<uint4*>(dst + g * 8) = ov;
                             }
                         }
+                    }
+                }
+            } else if (EPI == EPI_PARTIAL) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    float v[32];
+                    tmem_ld32(t_acc + c * 32, v);
+                    tmem_ld_wait();
+                    const int col0 = n_blk * BN + c * 32;
+                    if (row < p.M) {
+                        float* dst = p.partial + ((size_t)ks * p.M + row) * p.N + col0;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (col0 + g * 4 < p.N)           // N is a multiple of 8
+                                *reinterpret_cast<float4*>(dst + g * 4) =
+                                    make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
                     }
                 }
             } else if (EPI == EPI_SWIGLU) {
@@ -346,6 +374,38 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
     if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, 1);
+}
+
+// C = bf16( sum over K ranges of partial + residual ).  8 outputs per thread.
+__global__ void splitk_reduce_kernel(const float* __restrict__ partial, int split, const __nv_bfloat16* residual,
+                                     __nv_bfloat16* C, int M, int N) {
+    const size_t i8 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    const size_t total = (size_t)M * N;
+    if (i8 >= total) return;
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) x[j] = 0.f;
+    for (int s = 0; s < split; ++s) {
+        const float4 a = *reinterpret_cast<const float4*>(partial + s * total + i8);
+        const float4 b = *reinterpret_cast<const float4*>(partial + s * total + i8 + 4);
+        x[0] += a.x; x[1] += a.y; x[2] += a.z; x[3] += a.w;
+        x[4] += b.x; x[5] += b.y; x[6] += b.z; x[7] += b.w;
+    }
+    if (residual) {
+        const uint4 rv = *reinterpret_cast<const uint4*>(residual + i8);
+        const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __bfloat1622float2(r2[j]);
+            x[2 * j] += f.x;
+            x[2 * j + 1] += f.y;
+        }
+    }
+    uint4 ov;
+    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
+    *reinterpret_cast<uint4*>(C + i8) = ov;
 }
 
 }  // namespace jot

@@ -97,22 +97,53 @@ __global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_b
 
 // Rotate-half RoPE in place on the Q and K heads of qkv [B*L, (nq + 2 nkv) * hd], and transpose V into
 // vt [B, nkv, hd, Lp] (keys contiguous) for the P.V product.  cs = [max_seq, hd/2] (cos, sin) table.
-// grid = (B*L, nq + 2*nkv), block = hd/2 threads.
-__global__ void rope_vt_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ vt,
-                               const float2* __restrict__ cs, int L, int Lp, int nq, int nkv, int hd) {
-    const int row = blockIdx.x, head = blockIdx.y, j = threadIdx.x, half = hd >> 1;
-    const int pos = row % L, b = row / L;
-    __nv_bfloat16* base = qkv + (size_t)row * (nq + 2 * nkv) * hd + (size_t)head * hd;
+// grid = (ceil(L/32), nq + 2*nkv, B): one CTA per (32 positions, head); 256 threads; 16-byte accesses.
+template <int HD>
+__global__ void __launch_bounds__(256) rope_vt_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ vt,
+                                                      const float2* __restrict__ cs, int L, int Lp, int nq, int nkv) {
+    constexpr int HALF = HD / 2;
+    constexpr int TPP = HD / 16;                   // threads per position (8 pairs each)
+    const int pos0 = blockIdx.x * 32, head = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
+    const size_t row_stride = (size_t)(nq + 2 * nkv) * HD;
     if (head < nq + nkv) {
-        const float2 c = cs[(size_t)pos * half + j];
-        const float x0 = __bfloat162float(base[j]), x1 = __bfloat162float(base[j + half]);
-        base[j] = __float2bfloat16_rn(x0 * c.x - x1 * c.y);
-        base[j + half] = __float2bfloat16_rn(x1 * c.x + x0 * c.y);
+        const int pl = tid / TPP, j0 = (tid % TPP) * 8, pos = pos0 + pl;
+        if (pl < 32 && pos < L) {
+            __nv_bfloat16* base = qkv + ((size_t)b * L + pos) * row_stride + (size_t)head * HD;
+            uint4 lo = *reinterpret_cast<const uint4*>(base + j0), hi = *reinterpret_cast<const uint4*>(base + HALF + j0);
+            __nv_bfloat16* l8 = reinterpret_cast<__nv_bfloat16*>(&lo);
+            __nv_bfloat16* h8 = reinterpret_cast<__nv_bfloat16*>(&hi);
+            const float2* c = cs + (size_t)pos * HALF + j0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const float2 k = c[t];
+                const float x0 = __bfloat162float(l8[t]), x1 = __bfloat162float(h8[t]);
+                l8[t] = __float2bfloat16_rn(x0 * k.x - x1 * k.y);
+                h8[t] = __float2bfloat16_rn(x1 * k.x + x0 * k.y);
+            }
+            *reinterpret_cast<uint4*>(base + j0) = lo;
+            *reinterpret_cast<uint4*>(base + HALF + j0) = hi;
+        }
     } else {
+        __shared__ __align__(16) __nv_bfloat16 tile[32][HD + 8];
         const int kvh = head - nq - nkv;
-        __nv_bfloat16* dst = vt + ((size_t)(b * nkv + kvh) * hd) * Lp + pos;
-        dst[(size_t)j * Lp] = base[j];
-        dst[(size_t)(j + half) * Lp] = base[j + half];
+        for (int v = tid; v < 32 * (HD / 8); v += 256) {
+            const int pl = v / (HD / 8), c8 = (v % (HD / 8)) * 8, pos = pos0 + pl;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (pos < L)
+                val = *reinterpret_cast<const uint4*>(qkv + ((size_t)b * L + pos) * row_stride + (size_t)head * HD + c8);
+            *reinterpret_cast<uint4*>(&tile[pl][c8]) = val;
+        }
+        __syncthreads();
+        for (int v = tid; v < HD * 4; v += 256) {
+            const int d = v / 4, g8 = (v % 4) * 8;
+            if (pos0 + g8 < Lp) {
+                uint4 out;
+                __nv_bfloat16* o8 = reinterpret_cast<__nv_bfloat16*>(&out);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) o8[t] = tile[g8 + t][d];
+                *reinterpret_cast<uint4*>(vt + ((size_t)(b * nkv + kvh) * HD + d) * Lp + pos0 + g8) = out;
+            }
+        }
     }
 }
 

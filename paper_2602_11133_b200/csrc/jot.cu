@@ -143,7 +143,31 @@ int make_weight_maps(const DeviceInfo* di, WeightMaps* w, const void* ptr, int r
     return JOT_OK;
 }
 
-int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, int epi, GemmParams p, cudaStream_t st) {
+// Split-K factor for a plain projection: when 256-wide tiles leave most SMs idle, cut K into up to 4
+// ranges so that (tiles x ranges) still fits one wave.  Needs `scratch` for the fp32 partial sums.
+int pick_split(int M, int N, int K, int sms, size_t scratch_bytes) {
+    const long tiles = (long)((M + 127) / 128) * ((N + 255) / 256);
+    const int num_kb = (K + kBK - 1) / kBK;
+    int split = (int)(sms / tiles);
+    if (split > 4) split = 4;
+    while (split > 1 && (num_kb / split < 8 || (size_t)split * M * N * 4 > scratch_bytes)) --split;
+    return split < 1 ? 1 : split;
+}
+
+int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, int epi, GemmParams p, cudaStream_t st,
+             float* scratch = nullptr, size_t scratch_bytes = 0) {
+    if (epi == EPI_STORE && scratch) {
+        const int split = pick_split(p.M, p.N, p.K, di->sms, scratch_bytes);
+        if (split > 1) {
+            p.split_k = split;
+            p.partial = scratch;
+            const long items = (long)((p.M + 127) / 128) * ((p.N + 255) / 256) * split;
+            JOT_TRY((launch_gemm_t<256, EPI_PARTIAL>(p, tmA, w.m256, (int)items, st)));
+            const size_t n8 = (size_t)p.M * p.N / 8;
+            splitk_reduce_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(scratch, split, p.residual, p.C, p.M, p.N);
+            return launch_check();
+        }
+    }
     const int n_out = (epi == EPI_SWIGLU) ? p.N / 2 : p.N;
     int bn = pick_bn(p.M, epi == EPI_SWIGLU ? 2 * n_out : n_out, di->sms);
     const int bn_out = (epi == EPI_SWIGLU) ? bn / 2 : bn;
@@ -191,6 +215,7 @@ struct jot_model {
     __nv_bfloat16 *h, *a, *qkv, *vt, *attn, *act, *hsel;
     int32_t* rows;
     float4* partials;
+    float* splitk;
     int R_cap;
     int32_t* canvas;      // generate: tokens [max_batch * max_seq]
     float *g_top1, *g_top2, *g_sumexp;
@@ -242,9 +267,11 @@ struct ProfScope {
 };
 
 struct Layout {
-    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, partials, canvas, top1, top2, sumexp, argmax, state, params,
+    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, partials, splitk, canvas, top1, top2, sumexp, argmax, state, params,
         total;
 };
+
+constexpr size_t kSplitKBytes = (size_t)148 * 128 * 256 * 4 + 4096;   // one wave of 128 x 256 fp32 tiles
 
 bool config_ok(const jot_model_config* c) {
     if (!c) return false;
@@ -279,6 +306,7 @@ Layout make_layout(const jot_model_config* c, int max_batch, int max_seq) {
     l.hsel = take(R_cap * c->d_model * 2);
     l.rows = take(R_cap * 4);
     l.partials = take((size_t)256 * R_cap * sizeof(float4));   // up to 256 vocabulary chunks
+    l.splitk = take(kSplitKBytes);
     l.canvas = take(M * 4);
     l.top1 = take(M * 4);
     l.top2 = take(M * 4);
@@ -331,11 +359,13 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = qkv_cols; p.K = d; p.C = m->qkv; p.ldc = qkv_cols; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_QKV, st);
-            JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_STORE, p, st));
+            JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_STORE, p, st, m->splitk, kSplitKBytes));
         }
         {
             ProfScope ps(m, JOT_PROF_ROPE, st);
-            rope_vt_kernel<<<dim3(M, nq + 2 * nkv), hd / 2, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv, hd);
+            const dim3 rgrid((L + 31) / 32, nq + 2 * nkv, B);
+            if (hd == 128) rope_vt_kernel<128><<<rgrid, 256, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
+            else rope_vt_kernel<64><<<rgrid, 256, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
         }
         JOT_TRY(launch_check());
         AttnParams ap{};
@@ -351,7 +381,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = d; p.K = nq * hd; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_O, st);
-            JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st));
+            JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes));
         }
         {
             ProfScope ps(m, JOT_PROF_RMSNORM, st);
@@ -368,7 +398,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_DOWN, st);
-            JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st));
+            JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st, m->splitk, kSplitKBytes));
         }
     }
     return JOT_OK;
@@ -496,6 +526,7 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
     m->hsel = (__nv_bfloat16*)(base + lay.hsel);
     m->rows = (int32_t*)(base + lay.rows);
     m->partials = (float4*)(base + lay.partials);
+    m->splitk = (float*)(base + lay.splitk);
     m->R_cap = (int)align_up((size_t)max_batch * max_seq, 128);
     m->canvas = (int32_t*)(base + lay.canvas);
     m->g_top1 = (float*)(base + lay.top1);
@@ -707,7 +738,7 @@ int jot_profile_read(jot_model* m, double* ms, int64_t* launches, int n_classes)
 }
 
 int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
-                  int32_t* d_status, void* stream) {
+                  void* d_scratch, size_t scratch_bytes, int32_t* d_status, void* stream) {
     if (!d_A || !d_W || !d_C) return JOT_ERR_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return JOT_ERR_ARG;
     if (N % 8 || K % 8) return JOT_ERR_SHAPE;
@@ -723,7 +754,8 @@ int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void
     GemmParams p{};
     p.M = M; p.N = N; p.K = K; p.C = (__nv_bfloat16*)d_C; p.residual = (const __nv_bfloat16*)d_residual; p.ldc = N;
     p.status = d_status;
-    return run_gemm(di, tmA, wm, EPI_STORE, p, (cudaStream_t)stream);
+    if (d_scratch && (reinterpret_cast<uintptr_t>(d_scratch) & 15)) return JOT_ERR_ARG;
+    return run_gemm(di, tmA, wm, EPI_STORE, p, (cudaStream_t)stream, (float*)d_scratch, d_scratch ? scratch_bytes : 0);
 }
 
 }  // extern "C"

@@ -90,7 +90,7 @@ def _lib():
                                      C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32),
                                      C.POINTER(C.c_int32), C.c_void_p]
         lib.jot_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
-                                      C.c_void_p, C.c_void_p]
+                                      C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         lib.jot_launch_count.restype = C.c_int64
         lib.jot_profile.argtypes = [C.c_void_p, C.c_int]
         lib.jot_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int]
@@ -251,14 +251,16 @@ def accept_freeze(params: Params, mask_id: int, tokens: torch.Tensor, blk_lo: in
 
 
 def gemm_bf16(a: torch.Tensor, w: torch.Tensor, residual: Optional[torch.Tensor] = None,
-              out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """out[M, N] = a[M, K] @ w[N, K]^T (+ residual), bf16 in/out, fp32 accumulate."""
+              out: Optional[torch.Tensor] = None, scratch: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """out[M, N] = a[M, K] @ w[N, K]^T (+ residual), bf16 in/out, fp32 accumulate.
+    scratch: optional float32 CUDA tensor the kernel may use for split-K partial sums."""
     M, K = a.shape
     N = w.shape[0]
     out = torch.empty(M, N, dtype=torch.bfloat16, device=a.device) if out is None else out
     status = torch.zeros(1, dtype=torch.int32, device=a.device)
     _check(_lib().jot_gemm_bf16(_ptr(a, torch.bfloat16, "a"), _ptr(w, torch.bfloat16, "w"),
                                 _ptr(residual, torch.bfloat16, "residual"), _ptr(out, torch.bfloat16, "out"), M, N, K,
+                                _ptr(scratch, torch.float32, "scratch"), scratch.numel() * 4 if scratch is not None else 0,
                                 status.data_ptr(), _stream()), "jot_gemm_bf16")
     if int(status.item()) != 0:
         raise JotError(-5, "jot_gemm_bf16")

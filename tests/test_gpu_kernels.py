@@ -43,6 +43,23 @@ def test_gemm_matches_float64_definition(jot, M, N, K, with_res):
     assert got.abs().max().item() > 0.1
 
 
+@pytest.mark.parametrize("M,N,K", [(384, 4096, 4096), (384, 4096, 12288), (200, 512, 2048), (96, 264, 1096)])
+@pytest.mark.parametrize("with_res", [False, True])
+def test_gemm_split_k_matches_float64_definition(jot, M, N, K, with_res):
+    """Few output tiles and a long K: the kernel cuts K into ranges and a second kernel adds them."""
+    a = inputs.normal(4, "a", (M, K), 1.0).cuda()
+    w = inputs.normal(4, "w", (N, K), 0.03).cuda()
+    res = inputs.normal(4, "r", (M, N), 1.0).cuda() if with_res else None
+    scratch = torch.empty(4 * M * N, dtype=torch.float32, device="cuda")
+    n0 = jot.launch_count()
+    out = jot.gemm_bf16(a, w, res, scratch=scratch)
+    assert jot.launch_count() - n0 == 2          # partial-sum kernel + reduction: the split path really ran
+    want = bf16_matmul_oracle(a.cpu(), w.cpu(), None if res is None else res.cpu())
+    err = (out.cpu().double() - want).abs()
+    tol = 2.0 ** -8 * want.abs() + 1e-3 * want.abs().max()
+    assert (err <= tol).all(), f"max err {err.max().item()}"
+
+
 def test_gemm_residual_in_place(jot):
     a = inputs.normal(2, "a", (384, 512), 1.0).cuda()
     w = inputs.normal(2, "w", (1024, 512), 0.05).cuda()
