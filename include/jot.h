@@ -34,7 +34,8 @@ typedef enum {
     JOT_ERR_WORKSPACE = -3,  /* workspace missing, misaligned or smaller than required        */
     JOT_ERR_CUDA = -4,       /* a CUDA runtime/driver call failed: see jot_last_cuda_error()  */
     JOT_ERR_TIMEOUT = -5,    /* a bounded device-side wait expired; outputs are undefined     */
-    JOT_ERR_DEVICE = -6      /* not an sm_100 device, or the driver lacks tensor-map support  */
+    JOT_ERR_DEVICE = -6,     /* not an sm_100 device, or the driver lacks tensor-map support  */
+    JOT_ERR_LIMIT = -7       /* larger than the built-in scratch of jot_gemm_bf16_noalloc     */
 } jot_status;
 
 /* Static message for a status code. */
@@ -166,6 +167,28 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
  * d_status: device int32 the kernel sets non-zero if a bounded wait expires (may be NULL). */
 int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
                   void* d_scratch, size_t scratch_bytes, int32_t* d_status, void* stream);
+
+/* jot_gemm_bf16 for callers that must not allocate device memory.  (The paper has no counterpart
+ * to this function; it exists for the library's users.)  Some code that wants this projection runs
+ * where cudaMalloc is off limits: inside a latency-critical serving loop whose memory was carved up at
+ * start-up, under a framework whose caching allocator must stay the only owner of the device heap, or
+ * in a plugin that is handed buffers and forbidden to create its own.  jot_gemm_bf16 makes such a
+ * caller bring scratch for the split-K partial sums; this variant brings its own: a fixed array of
+ * JOT_NOALLOC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the library
+ * holds that much memory until the process exits.  Arguments and result are those of jot_gemm_bf16
+ * without the scratch pair; inputs and outputs are still the caller's.
+ *   - Limit: 4 * M * N * sizeof(float) must fit in the array (M * N <= 1,048,576), else JOT_ERR_LIMIT
+ *     and nothing is launched.
+ *   - The first call on each device looks up the array's device address (a host-side query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - No cudaMalloc/cudaFree and no allocating library routine is called, on any call.
+ *   - All calls share the one array and it keeps whatever the previous call left there.  Nothing in it
+ *     needs to start at zero: every partial sum the reduction reads is written earlier in the same
+ *     call.  Two calls whose kernels overlap on the GPU (different streams, or different host threads
+ *     on different streams) race on it; issue them on one stream or serialise them yourself. */
+#define JOT_NOALLOC_SCRATCH_BYTES (16u << 20)
+int jot_gemm_bf16_noalloc(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N, int K,
+                          int32_t* d_status, void* stream);
 
 /* Optional timing of the kernels a model launches, by class, with CUDA events recorded on the launching
  * stream around each launch.  jot_profile(m, 1) starts (and clears) the accumulation, jot_profile(m, 0)

@@ -8,6 +8,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -479,6 +480,7 @@ const char* jot_status_string(int s) {
         case JOT_ERR_CUDA: return "CUDA call failed";
         case JOT_ERR_TIMEOUT: return "bounded device wait expired";
         case JOT_ERR_DEVICE: return "device or driver not supported (needs sm_100 and tensor-map support)";
+        case JOT_ERR_LIMIT: return "problem larger than the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
@@ -759,3 +761,54 @@ int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------- projection without any allocation
+// Split-K needs room for its fp32 partial sums.  Here that room is a fixed array that is part of the
+// library image: every GPU that loads the library carries these 16 MiB until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[JOT_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_noalloc_mu;
+float* g_noalloc_ptr[64] = {};
+
+// The array's name is only a handle on the host side; its device address has to be asked for, once
+// per device, with that device current.
+int noalloc_scratch_address(float** out) {
+    int dev = 0;
+    JOT_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return JOT_ERR_DEVICE;
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        JOT_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        if (!ptr) return JOT_ERR_DEVICE;
+        g_noalloc_ptr[dev] = static_cast<float*>(ptr);
+    }
+    *out = g_noalloc_ptr[dev];
+    return JOT_OK;
+}
+}  // namespace
+
+extern "C" int jot_gemm_bf16_noalloc(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N,
+                                     int K, int32_t* d_status, void* stream) {
+    if (!d_A || !d_W || !d_C) return JOT_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return JOT_ERR_ARG;
+    if (N % 8 || K % 8) return JOT_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_A) | reinterpret_cast<uintptr_t>(d_W) | reinterpret_cast<uintptr_t>(d_C) |
+         reinterpret_cast<uintptr_t>(d_residual)) & 15)
+        return JOT_ERR_ARG;
+    // room for four K ranges of the whole output, whatever split the kernel then picks
+    if ((size_t)M * (size_t)N * 4 * sizeof(float) > (size_t)JOT_NOALLOC_SCRATCH_BYTES) return JOT_ERR_LIMIT;
+    DeviceInfo* di = nullptr;
+    JOT_TRY(device_info(&di));
+    float* scratch = nullptr;
+    JOT_TRY(noalloc_scratch_address(&scratch));
+    CUtensorMap tmA;
+    WeightMaps wm;
+    JOT_TRY(make_map_2d(di, &tmA, d_A, M, K, K, 128));
+    JOT_TRY(make_weight_maps(di, &wm, d_W, N, K, false));
+    GemmParams p{};
+    p.M = M; p.N = N; p.K = K; p.C = (__nv_bfloat16*)d_C; p.residual = (const __nv_bfloat16*)d_residual; p.ldc = N;
+    p.status = d_status;
+    return run_gemm(di, tmA, wm, EPI_STORE, p, (cudaStream_t)stream, scratch, (size_t)JOT_NOALLOC_SCRATCH_BYTES);
+}

@@ -19,8 +19,10 @@ LIB_PATH = os.path.join(_HERE, "libjot.so")
 EXPORTS = [
     "jot_status_string", "jot_last_cuda_error", "jot_workspace_bytes", "jot_init_model", "jot_free_model",
     "jot_denoise_step", "jot_lm_head_stats", "jot_accept_freeze", "jot_generate", "jot_gemm_bf16",
-    "jot_launch_count", "jot_profile", "jot_profile_read",
+    "jot_launch_count", "jot_profile", "jot_profile_read", "jot_gemm_bf16_noalloc",
 ]
+
+NOALLOC_SCRATCH_BYTES = 16 << 20
 
 PROF_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "rows",
                 "lm_head", "merge", "accept"]
@@ -91,6 +93,8 @@ def _lib():
                                      C.POINTER(C.c_int32), C.c_void_p]
         lib.jot_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                       C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        lib.jot_gemm_bf16_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                              C.c_void_p, C.c_void_p]
         lib.jot_launch_count.restype = C.c_int64
         lib.jot_profile.argtypes = [C.c_void_p, C.c_int]
         lib.jot_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int]
@@ -264,4 +268,21 @@ def gemm_bf16(a: torch.Tensor, w: torch.Tensor, residual: Optional[torch.Tensor]
                                 status.data_ptr(), _stream()), "jot_gemm_bf16")
     if int(status.item()) != 0:
         raise JotError(-5, "jot_gemm_bf16")
+    return out
+
+
+def gemm_bf16_noalloc(a: torch.Tensor, w: torch.Tensor, residual: Optional[torch.Tensor], out: torch.Tensor,
+                      status: torch.Tensor) -> torch.Tensor:
+    """out[M, N] = a[M, K] @ w[N, K]^T (+ residual) through the entry point that never allocates.
+
+    For callers that may not create device memory (a serving loop with a fixed memory plan, a plugin that
+    only gets buffers handed to it): the split-K scratch is a fixed 16 MiB array inside the library, so
+    4 * M * N * 4 bytes must fit in it.  `out` and the int32 `status` word are the caller's, too; this
+    wrapper creates no tensor.  Calls share the array: keep them on one stream."""
+    M, K = a.shape
+    N = w.shape[0]
+    _check(_lib().jot_gemm_bf16_noalloc(_ptr(a, torch.bfloat16, "a"), _ptr(w, torch.bfloat16, "w"),
+                                        _ptr(residual, torch.bfloat16, "residual"), _ptr(out, torch.bfloat16, "out"),
+                                        M, N, K, _ptr(status, torch.int32, "status"), _stream()),
+           "jot_gemm_bf16_noalloc")
     return out
