@@ -18,6 +18,14 @@ namespace jot {
 
 enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2, EPI_PARTIAL = 3 };
 
+// Pipeline depth (shared-memory stages of one A tile + one W tile); both fill ~192 KB.
+#ifndef JOT_GEMM_STAGES_256
+#define JOT_GEMM_STAGES_256 4
+#endif
+#ifndef JOT_GEMM_STAGES_128
+#define JOT_GEMM_STAGES_128 6
+#endif
+
 constexpr int kBM = 128;          // rows per tile = TMEM lanes
 constexpr int kBK = 64;           // bf16 elements per 128-byte swizzled smem row
 constexpr int kGemmThreads = 192;
@@ -45,7 +53,7 @@ struct GemmSmem {
     static constexpr int A_BYTES = kBM * kBK * 2;
     static constexpr int B_BYTES = BN * kBK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 256) ? 4 : 6;
+    static constexpr int STAGES = (BN == 256) ? JOT_GEMM_STAGES_256 : JOT_GEMM_STAGES_128;
     static constexpr int DYN_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align to 1024
 };
 

@@ -188,35 +188,55 @@ __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restr
     if (tid == 0) *d_R = total;
 }
 
-// Merge the per-chunk partial statistics of each active row (chunks ascend through the vocabulary, so
-// "strictly greater" keeps the lowest index on ties) and scatter them to the [B, L] outputs.
-__global__ void merge_stats_kernel(const float4* __restrict__ partials, int R_pad, int grid_gemm, int n_vt,
-                                   const int32_t* __restrict__ rows, const int32_t* __restrict__ d_R,
-                                   float* __restrict__ top1, float* __restrict__ top2, float* __restrict__ sumexp,
-                                   int32_t* __restrict__ argmax) {
+// Merge the per-chunk partial statistics of each active row and scatter them to the [B, L] outputs.
+// The merge is associative and symmetric (equal maxima resolve to the lower token id), so one warp per
+// row lets its lanes take chunks round-robin and then combines them with a butterfly.
+struct StatTuple {
+    float m1, m2, S;
+    int i1;
+};
+__device__ __forceinline__ StatTuple merge_tuples(const StatTuple& a, const StatTuple& b) {
+    StatTuple r;
+    r.m1 = fmaxf(a.m1, b.m1);
+    r.m2 = fmaxf(fmaxf(a.m2, b.m2), fminf(a.m1, b.m1));
+    const float sa = (a.m1 == -INFINITY) ? 0.f : a.S * expf(a.m1 - r.m1);
+    const float sb = (b.m1 == -INFINITY) ? 0.f : b.S * expf(b.m1 - r.m1);
+    r.S = sa + sb;
+    r.i1 = (b.m1 > a.m1 || (b.m1 == a.m1 && b.i1 < a.i1)) ? b.i1 : a.i1;
+    return r;
+}
+__global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restrict__ partials, int R_pad, int grid_gemm,
+                                                          int n_vt, const int32_t* __restrict__ rows,
+                                                          const int32_t* __restrict__ d_R, float* __restrict__ top1,
+                                                          float* __restrict__ top2, float* __restrict__ sumexp,
+                                                          int32_t* __restrict__ argmax) {
     const int R = *d_R;
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= R) return;
-    int n_rb = (R + 127) / 128;
+    const int n_rb = (R + 127) / 128;
     int n_ch = grid_gemm / n_rb;
     if (n_ch > n_vt) n_ch = n_vt;
-    float m1 = -INFINITY, m2 = -INFINITY, S = 0.f;
-    int i1 = 0x7fffffff;
-    for (int c = 0; c < n_ch; ++c) {
-        const float4 t = partials[(size_t)c * R_pad + r];
-        const float bm1 = t.x, bm2 = t.z, bS = t.w;
-        const int bi1 = __float_as_int(t.y);
-        const float nm = fmaxf(m1, bm1);
-        m2 = fmaxf(fmaxf(m2, bm2), fminf(m1, bm1));
-        S = S * expf(m1 - nm) + bS * expf(bm1 - nm);
-        if (bm1 > m1) i1 = bi1;
-        m1 = nm;
+    StatTuple t{-INFINITY, -INFINITY, 0.f, 0x7fffffff};
+    for (int c = lane; c < n_ch; c += 32) {
+        const float4 v = partials[(size_t)c * R_pad + r];
+        t = merge_tuples(t, StatTuple{v.x, v.z, v.w, __float_as_int(v.y)});
     }
-    const int flat = rows[r];
-    top1[flat] = m1;
-    top2[flat] = m2;
-    sumexp[flat] = S;
-    argmax[flat] = i1;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        StatTuple u;
+        u.m1 = __shfl_xor_sync(0xffffffffu, t.m1, o);
+        u.m2 = __shfl_xor_sync(0xffffffffu, t.m2, o);
+        u.S = __shfl_xor_sync(0xffffffffu, t.S, o);
+        u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+        t = merge_tuples(t, u);
+    }
+    if (lane == 0) {
+        const int flat = rows[r];
+        top1[flat] = t.m1;
+        top2[flat] = t.m2;
+        sumexp[flat] = t.S;
+        argmax[flat] = t.i1;
+    }
 }
 
 // x = [prompt ; mask_id * G]  and fresh loop state  (Algorithm 1, initialisation)

@@ -424,7 +424,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     }
     const int n_vt = (c.vocab + bn - 1) / bn;
     ProfScope ps(m, JOT_PROF_MERGE, st);
-    merge_stats_kernel<<<(m->R_cap + 127) / 128, 128, 0, st>>>(m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
+    merge_stats_kernel<<<(M + 3) / 4, 128, 0, st>>>(m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
                                                                top1, top2, sumexp, argmax);
     return launch_check();
 }

@@ -23,17 +23,25 @@ def oracle_stats_for_rows(logits_rows: torch.Tensor, mask_id) -> List[jo.RowStat
     return [jo.row_stats(logits_rows[r].numpy(), mask_id) for r in range(logits_rows.shape[0])]
 
 
-def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowStats], rel=REL_TOL):
-    """Returns (n_checked, n_near_tie).  Raises AssertionError on a real mismatch."""
+def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowStats], rel=REL_TOL,
+                  gap_from_tolerance=False):
+    """Returns (n_checked, n_near_tie).  Raises AssertionError on a real mismatch.
+
+    The argmax must agree unless the oracle's top-2 gap is below GAP_TOL.  With gap_from_tolerance (deep
+    models, where the bf16 path's logit noise is far above 1e-3) the exemption is the one the logit
+    tolerance itself implies: two logits that may each move by rel*scale can swap when their gap is below
+    2*rel*scale.  Exempt rows are counted, and their argmax must still be the oracle's runner-up region:
+    the GPU's top-1 logit has to be within tolerance of the oracle's."""
     near = 0
     for r, st in enumerate(want):
         scale = max(abs(st.m1), abs(st.m2), 1.0)
+        gap_tol = max(GAP_TOL, 2 * rel * scale) if gap_from_tolerance else GAP_TOL
         assert abs(got_top1[r] - st.m1) <= rel * scale, (r, got_top1[r], st.m1)
         assert abs(got_top2[r] - st.m2) <= rel * scale, (r, got_top2[r], st.m2)
         # log-sum-exp agrees to the logit tolerance  <=> S agrees to a relative factor
         assert abs(math.log(got_sumexp[r]) - math.log(st.S)) <= rel * scale, (r, got_sumexp[r], st.S)
-        if st.m1 - st.m2 < GAP_TOL:
-            near += 1                     # top-2 gap below 1e-3: either index is a valid argmax
+        if st.m1 - st.m2 < gap_tol:
+            near += 1                     # top-2 gap inside the margin: either index is a valid argmax
         else:
             assert int(got_argmax[r]) == st.i1, (r, int(got_argmax[r]), st.i1, st.m1 - st.m2)
     return len(want), near
