@@ -160,16 +160,27 @@ def time_oracle_sample(g, w_any, nl, B, P, G, block_len, params, sample_layers=2
 
 # ------------------------------------------------------------------------------------------------ main
 def dist_setup(world, dev):
+    """One process per GPU; the process group only carries the timing barrier and the max over ranks
+    (replicas are independent: there is no collective on the data path)."""
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+        if dev.type == "cuda":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group("gloo")
 
 
 def barrier(world):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
+
+
+def aggregate_rate(units_per_rank, world, ms_max):
+    """Whole-job rate: what all ranks processed divided by the slowest rank's time."""
+    return world * units_per_rank / (ms_max / 1e3)
 
 
 def max_over_ranks(values, world, dev):
@@ -345,7 +356,7 @@ def run_model(args, jot, dev, world, rank, peaks, peaks_kind, config, g, nl, B, 
              "weight_stream_gbs": round(weight_bytes(g, nl) / step_s / 1e9, 1),
              "hbm_frac": round(weight_bytes(g, nl) / step_s / 1e9 / peaks.get("hbm_gbs", 6650.0), 4),
              "of": peaks_kind}
-    line = base_line(args, world, "denoising_steps_per_s", "steps/s", world * args.steps / (ms_max / 1e3),
+    line = base_line(args, world, "denoising_steps_per_s", "steps/s", aggregate_rate(args.steps, world, ms_max),
                      ms_max / args.steps, config, clocks, launches)
     line["generated_tokens_per_s"] = round(world * B * (host_out.shape[1] - P) / (e2e_ms_max / 1e3), 2)
     line["e2e"] = {"value": round(world * passes / (e2e_ms_max / 1e3), 3), "unit": "steps/s",
@@ -435,7 +446,7 @@ def run_lmhead(args, jot, dev, world, rank, peaks, peaks_kind, config, g, nl, B,
     roofline["active_rows"] = R
     roofline["frac_of_burst"] = round(roofline["achieved"] / peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]), 4) \
         if roofline.get("bound") == "tensor" else None
-    line = base_line(args, world, "lm_head_accept_steps_per_s", "steps/s", world * args.steps / (ms_max / 1e3),
+    line = base_line(args, world, "lm_head_accept_steps_per_s", "steps/s", aggregate_rate(args.steps, world, ms_max),
                      ms_max / args.steps, config, clocks, launches)
     line["active_rows_per_s"] = round(world * R * args.steps / (ms_max / 1e3), 1)
     line["e2e"] = {"value": round(world / (e2e_ms_max / 1e3), 3), "unit": "steps/s",
