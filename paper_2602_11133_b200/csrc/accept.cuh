@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "pdl.cuh"
+
 namespace jot {
 
 constexpr int kAcceptThreads = 256;
@@ -52,6 +54,8 @@ struct AcceptArgs {
 // Dynamic shared memory: resolved bitmap words, candidate list, candidate sum-exp, candidate flags.
 __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const AcceptArgs a) {
     extern __shared__ uint32_t sh[];
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int L = a.L, b = blockIdx.x, tid = threadIdx.x;
     const int n_words = (L + 31) / 32;
     uint32_t* res_bits = sh;                                   // [n_words + 2] resolved bitmap (padded)

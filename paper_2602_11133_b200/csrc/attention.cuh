@@ -15,6 +15,7 @@
 // block never reads across a sequence boundary: out-of-range positions read as zero); V transposed
 // vt [B * nkv * hd, Lp] with keys contiguous, so that both products take K-major operands.
 #pragma once
+#include "pdl.cuh"
 #include "ptx.cuh"
 
 namespace jot {
@@ -95,6 +96,8 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
+    grid_launch_dependents();
+    grid_dependency_wait();
 
     if (warp == 0) {
         if (lane == 0) {

@@ -12,6 +12,7 @@
 //        EPI_PARTIAL fp32 partial sums of one K range (split-K for projections with too few output
 //                    tiles to fill the SMs); splitk_reduce_kernel adds the ranges and the residual
 #pragma once
+#include "pdl.cuh"
 #include "ptx.cuh"
 
 namespace jot {
@@ -84,6 +85,36 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (p.K + kBK - 1) / kBK;
 
+    // ---- setup ----
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 4);
+        }
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(&tmem_base_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    // everything above is on-chip; from here on global memory written by earlier kernels is read
+    grid_launch_dependents();
+    grid_dependency_wait();
+
+
     // ---- tile schedule (identical in every role) ----
     int m_blk0 = 0, n_first = 0, n_count = 0;      // EPI_STATS: one row block, a range of vocabulary tiles
     int num_m = (p.M + kBM - 1) / kBM;
@@ -126,32 +157,6 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         n_blk = t / num_m;
         return true;
     };
-
-    // ---- setup ----
-    if (threadIdx.x == 0) {
-        abort_flag = 0;
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 1);
-        }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(&acc_full[a], 1);
-            mbar_init(&acc_empty[a], 4);
-        }
-        fence_barrier_init();
-        fence_proxy_async_smem();
-        tma_prefetch_desc(&tmA);
-        tma_prefetch_desc(&tmB);
-    }
-    if (warp == 1) {
-        tmem_alloc(&tmem_base_slot, TMEM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = tmem_base_slot;
-    volatile int* abortp = &abort_flag;
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -387,6 +392,8 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
 // C = bf16( sum over K ranges of partial + residual ).  8 outputs per thread.
 __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int split, const __nv_bfloat16* residual,
                                      __nv_bfloat16* C, int M, int N) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const size_t i8 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
     const size_t total = (size_t)M * N;
     if (i8 >= total) return;

@@ -36,6 +36,8 @@ __device__ __forceinline__ float block_sum(float v, float* scratch /* >= 33 floa
 // h[row, :] = E[tokens[row], :]          one CTA per row, 16-byte copies (d multiple of 8)
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E,
                              __nv_bfloat16* __restrict__ h, int d) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int row = blockIdx.x;
     const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[row] * d);
     uint4* dst = reinterpret_cast<uint4*>(h + (size_t)row * d);
@@ -48,6 +50,8 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bflo
 __global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
                                __nv_bfloat16* __restrict__ out, int d, float eps, const int32_t* __restrict__ rows,
                                const int32_t* __restrict__ d_R) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     __shared__ float scratch[33];
     const int r = blockIdx.x;
     int src = r;
@@ -101,6 +105,8 @@ __global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_b
 template <int HD>
 __global__ void __launch_bounds__(256) rope_vt_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ vt,
                                                       const float2* __restrict__ cs, int L, int Lp, int nq, int nkv) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     constexpr int HALF = HD / 2;
     constexpr int TPP = HD / 16;                   // threads per position (8 pairs each)
     const int pos0 = blockIdx.x * 32, head = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
@@ -154,6 +160,8 @@ __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restr
                                                           const SeqState* __restrict__ state, int P, int block_len,
                                                           int n_blocks, int32_t* __restrict__ rows,
                                                           int32_t* __restrict__ d_R) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     __shared__ int warp_counts[32];
     __shared__ int total;
     const int tid = threadIdx.x, wid = tid >> 5, ln = tid & 31;
@@ -210,6 +218,8 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
                                                           const int32_t* __restrict__ d_R, float* __restrict__ top1,
                                                           float* __restrict__ top2, float* __restrict__ sumexp,
                                                           int32_t* __restrict__ argmax) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int R = *d_R;
     const int r = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= R) return;
@@ -242,6 +252,8 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
 // x = [prompt ; mask_id * G]  and fresh loop state  (Algorithm 1, initialisation)
 __global__ void init_canvas_kernel(const int32_t* __restrict__ prompt, int32_t* __restrict__ x, int B, int P, int G,
                                    int32_t mask_id, SeqState* __restrict__ state) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int L = P + G;
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < B * L) {

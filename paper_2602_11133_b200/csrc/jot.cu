@@ -49,6 +49,23 @@ inline int launch_check() {
     return JOT_OK;
 }
 
+// Every kernel goes out through here: programmatic stream serialization lets a kernel's launch and
+// on-chip prologue overlap the tail of its predecessor (see pdl.cuh for the device side).
+template <typename... KArgs, typename... Args>
+void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);     // errors are picked up by launch_check()
+}
+
 // ---------------------------------------------------------------- device facts
 struct DeviceInfo {
     int ok = 0, sms = 0, status = JOT_OK;
@@ -121,7 +138,7 @@ int launch_gemm_t(const GemmParams& p, const CUtensorMap& tmA, const CUtensorMap
                                       GemmSmem<BN>::DYN_BYTES));
         attr_set[dev & 63] = true;
     }
-    gemm_kernel<BN, EPI><<<grid, kGemmThreads, GemmSmem<BN>::DYN_BYTES, st>>>(p, tmA, tmB);
+    launch_k((gemm_kernel<BN, EPI>), dim3(grid), dim3(kGemmThreads), GemmSmem<BN>::DYN_BYTES, st, p, tmA, tmB);
     return launch_check();
 }
 
@@ -165,7 +182,7 @@ int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, 
             const long items = (long)((p.M + 127) / 128) * ((p.N + 255) / 256) * split;
             JOT_TRY((launch_gemm_t<256, EPI_PARTIAL>(p, tmA, w.m256, (int)items, st)));
             const size_t n8 = (size_t)p.M * p.N / 8;
-            splitk_reduce_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(scratch, split, p.residual, p.C, p.M, p.N);
+            launch_k(splitk_reduce_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), 0, st, scratch, split, p.residual, p.C, p.M, p.N);
             return launch_check();
         }
     }
@@ -192,7 +209,7 @@ int launch_attention_t(const AttnParams& p, const CUtensorMap& tq, const CUtenso
                                       AttnSmem<HD>::DYN_BYTES));
         attr_set[dev & 63] = true;
     }
-    attention_kernel<HD><<<grid, kAttnThreads, AttnSmem<HD>::DYN_BYTES, st>>>(p, tq, tv);
+    launch_k((attention_kernel<HD>), dim3(grid), dim3(kAttnThreads), AttnSmem<HD>::DYN_BYTES, st, p, tq, tv);
     return launch_check();
 }
 
@@ -347,13 +364,13 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
 
     {
         ProfScope ps(m, JOT_PROF_EMBED, st);
-        embed_kernel<<<M, 128, 0, st>>>(d_tokens, m->embed, m->h, d);
+        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d);
     }
     JOT_TRY(launch_check());
     for (int l = 0; l < c.n_layers; ++l) {
         {
             ProfScope ps(m, JOT_PROF_RMSNORM, st);
-            rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->attn_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+            launch_k(rmsnorm_kernel, dim3(M), dim3(256), 0, st, m->h, m->attn_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
         }
         JOT_TRY(launch_check());
         GemmParams p{};
@@ -365,8 +382,8 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         {
             ProfScope ps(m, JOT_PROF_ROPE, st);
             const dim3 rgrid((L + 31) / 32, nq + 2 * nkv, B);
-            if (hd == 128) rope_vt_kernel<128><<<rgrid, 256, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
-            else rope_vt_kernel<64><<<rgrid, 256, 0, st>>>(m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
+            if (hd == 128) launch_k((rope_vt_kernel<128>), dim3(rgrid), dim3(256), 0, st, m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
+            else launch_k((rope_vt_kernel<64>), dim3(rgrid), dim3(256), 0, st, m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
         }
         JOT_TRY(launch_check());
         AttnParams ap{};
@@ -386,7 +403,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         }
         {
             ProfScope ps(m, JOT_PROF_RMSNORM, st);
-            rmsnorm_kernel<<<M, 256, 0, st>>>(m->h, m->mlp_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+            launch_k(rmsnorm_kernel, dim3(M), dim3(256), 0, st, m->h, m->mlp_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
         }
         JOT_TRY(launch_check());
         p = GemmParams{};
@@ -424,7 +441,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     }
     const int n_vt = (c.vocab + bn - 1) / bn;
     ProfScope ps(m, JOT_PROF_MERGE, st);
-    merge_stats_kernel<<<(M + 3) / 4, 128, 0, st>>>(m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
+    launch_k(merge_stats_kernel, dim3((M + 3) / 4), dim3(128), 0, st, m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
                                                                top1, top2, sumexp, argmax);
     return launch_check();
 }
@@ -432,6 +449,8 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
 // copy rows of a [*, d] bf16 matrix selected by `rows` (only r < *d_R)
 __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int d,
                                    const int32_t* __restrict__ rows, const int32_t* __restrict__ d_R) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int r = blockIdx.x;
     if (r >= *d_R) return;
     const uint4* s = reinterpret_cast<const uint4*>(src + (size_t)rows[r] * d);
@@ -460,7 +479,7 @@ int launch_accept(const AcceptArgs& a, cudaStream_t st) {
     if (smem > 48 * 1024) {
         JOT_CUDA(cudaFuncSetAttribute(accept_freeze_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
-    accept_freeze_kernel<<<a.B, kAcceptThreads, smem, st>>>(a);
+    launch_k(accept_freeze_kernel, dim3(a.B), dim3(kAcceptThreads), smem, st, a);
     return launch_check();
 }
 
@@ -599,10 +618,10 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
     JOT_TRY(encode_activation_maps(m, B, L));
     {
         ProfScope ps(m, JOT_PROF_ROWS, st);
-        build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+        launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
                                               m->ctrl + 1);
         JOT_TRY(launch_check());
-        gather_rows_kernel<<<B * L, 128, 0, st>>>((const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
+        launch_k(gather_rows_kernel, dim3(B * L), dim3(128), 0, st, (const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
                                                   m->ctrl + 1);
         JOT_TRY(launch_check());
     }
@@ -619,10 +638,10 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
     JOT_TRY(forward_body(m, d_tokens, B, L, st));
     {
         ProfScope ps(m, JOT_PROF_ROWS, st);
-        build_rows_kernel<<<1, 1024, 0, st>>>(d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+        launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
                                               m->ctrl + 1);
         JOT_TRY(launch_check());
-        rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
+        launch_k(rmsnorm_kernel, dim3(B * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
                                               m->ctrl + 1);
         JOT_TRY(launch_check());
     }
@@ -671,7 +690,7 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     cudaStream_t st = (cudaStream_t)stream;
     static_assert(sizeof(AcceptParamsDev) == sizeof(jot_params), "parameter struct layouts must agree");
     JOT_CUDA(cudaMemcpyAsync(m->params_dev, params, (size_t)n_par * sizeof(jot_params), cudaMemcpyHostToDevice, st));
-    init_canvas_kernel<<<(B * L + 255) / 256, 256, 0, st>>>(d_prompt, m->canvas, B, P, gen->gen_len, m->cfg.mask_id,
+    launch_k(init_canvas_kernel, dim3((B * L + 255) / 256), dim3(256), 0, st, d_prompt, m->canvas, B, P, gen->gen_len, m->cfg.mask_id,
                                                            m->state);
     JOT_TRY(launch_check());
     int passes = 0;
@@ -680,10 +699,10 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         JOT_TRY(forward_body(m, m->canvas, B, L, st));
         {
             ProfScope ps(m, JOT_PROF_ROWS, st);
-            build_rows_kernel<<<1, 1024, 0, st>>>(m->canvas, B, L, m->cfg.mask_id, 0, 0, m->state, P, gen->block_len,
+            launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, m->canvas, B, L, m->cfg.mask_id, 0, 0, m->state, P, gen->block_len,
                                                   nb, m->rows, m->ctrl + 1);
             JOT_TRY(launch_check());
-            rmsnorm_kernel<<<B * L, 256, 0, st>>>(m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps,
+            launch_k(rmsnorm_kernel, dim3(B * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps,
                                                   m->rows, m->ctrl + 1);
             JOT_TRY(launch_check());
         }
