@@ -9,6 +9,9 @@
 //        EPI_SWIGLU  bf16(silu(gate) * up), gate/up from the two halves of W -> C[M, N/2]
 //        EPI_STATS   online (max, argmax, runner-up, sum-exp) per row over a range of vocabulary tiles;
 //                    the logits are never written (LM head of the denoising step)
+//        EPI_QKV     QKV projection: bf16(acc), then rotary embedding on the Q and K heads (rotate-half,
+//                    table lookup by canvas position) written to C, and the V heads written transposed
+//                    (keys contiguous) for the attention kernel's P.V product
 //        EPI_PARTIAL fp32 partial sums of one K range (split-K for projections with too few output
 //                    tiles to fill the SMs); splitk_reduce_kernel adds the ranges and the residual
 #pragma once
@@ -17,7 +20,7 @@
 
 namespace jot {
 
-enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2, EPI_PARTIAL = 3 };
+enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2, EPI_PARTIAL = 3, EPI_QKV = 4 };
 
 // Pipeline depth (shared-memory stages of one A tile + one W tile); both fill ~192 KB.
 #ifndef JOT_GEMM_STAGES_256
@@ -39,6 +42,10 @@ struct GemmParams {
     int32_t* status;              // set non-zero when a bounded wait expired (nullable)
     int split_k;                  // EPI_PARTIAL: number of K ranges (>= 1); otherwise ignored
     float* partial;               // EPI_PARTIAL: [split_k][M][N] fp32
+    // EPI_QKV only: C = qkv [M, (nq + 2 nkv) * hd]; rows are (sequence, position) = (row / L, row % L)
+    __nv_bfloat16* vt;            // [B * nkv * hd, Lp] V transposed
+    const float2* rope_cs;        // [max_seq, hd / 2] (cos, sin)
+    int L, Lp, nq, nkv, hd;
     // EPI_STATS only
     const int32_t* d_R;           // number of active rows (device)
     const int32_t* rows;          // [R] flat canvas index b*L+i of each active row
@@ -276,6 +283,62 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
                                 *reinterpret_cast<uint4*>(dst + g * 8) = ov;
+                            }
+                        }
+                    }
+                }
+            } else if (EPI == EPI_QKV) {
+                const int hd = p.hd, half = hd >> 1;
+                const int seq = row / p.L, pos = row - seq * p.L;
+#pragma unroll 1
+                for (int hh = 0; hh < BN / hd; ++hh) {
+                    const int col_base = n_blk * BN + hh * hd;
+                    if (col_base >= p.N) break;
+                    const int head = col_base / hd;
+                    if (head < p.nq + p.nkv) {
+                        // rotate pairs (j, j + hd/2): 32 pairs at a time
+#pragma unroll 1
+                        for (int q = 0; q < half / 32; ++q) {
+                            float lo[32], hi[32];
+                            tmem_ld32(t_acc + hh * hd + q * 32, lo);
+                            tmem_ld32(t_acc + hh * hd + half + q * 32, hi);
+                            tmem_ld_wait();
+                            if (row < p.M) {
+                                const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cs + (size_t)pos * half + q * 32);
+                                __nv_bfloat16* dlo = p.C + (size_t)row * p.ldc + col_base + q * 32;
+                                __nv_bfloat16* dhi = dlo + half;
+#pragma unroll
+                                for (int g = 0; g < 4; ++g) {
+                                    uint4 olo, ohi;
+                                    __nv_bfloat162* l2 = reinterpret_cast<__nv_bfloat162*>(&olo);
+                                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&ohi);
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        const int e = g * 8 + 2 * j;
+                                        const float4 k = cs4[e >> 1];      // (cos, sin) of pairs e and e + 1
+                                        // the projection's output is bf16; the rotation acts on the rounded values
+                                        const float2 x0 = __bfloat1622float2(__floats2bfloat162_rn(lo[e], lo[e + 1]));
+                                        const float2 x1 = __bfloat1622float2(__floats2bfloat162_rn(hi[e], hi[e + 1]));
+                                        l2[j] = __floats2bfloat162_rn(x0.x * k.x - x1.x * k.y, x0.y * k.z - x1.y * k.w);
+                                        h2[j] = __floats2bfloat162_rn(x1.x * k.x + x0.x * k.y, x1.y * k.z + x0.y * k.w);
+                                    }
+                                    *reinterpret_cast<uint4*>(dlo + g * 8) = olo;
+                                    *reinterpret_cast<uint4*>(dhi + g * 8) = ohi;
+                                }
+                            }
+                        }
+                    } else {
+                        // V head: lane = position, so for a fixed d a warp writes 32 consecutive keys
+                        const int kvh = head - p.nq - p.nkv;
+#pragma unroll 1
+                        for (int c = 0; c < hd / 32; ++c) {
+                            float v[32];
+                            tmem_ld32(t_acc + hh * hd + c * 32, v);
+                            tmem_ld_wait();
+                            if (row < p.M) {
+                                __nv_bfloat16* dst = p.vt + ((size_t)(seq * p.nkv + kvh) * hd + c * 32) * p.Lp + pos;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) dst[(size_t)j * p.Lp] = __float2bfloat16_rn(v[j]);
                             }
                         }
                     }

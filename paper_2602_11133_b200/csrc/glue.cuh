@@ -1,5 +1,5 @@
 // Bandwidth-bound pieces of the denoising step: embedding gather, RMSNorm (plain and with active-row
-// compaction), rotary embedding + V transpose, active-row list, merge of the LM-head partial
+// compaction), split-K tail fused with the next norm, active-row list, merge of the LM-head partial
 // statistics, canvas initialisation.  All bf16 activations, fp32 arithmetic, 16-byte accesses.
 #pragma once
 #include <cuda_bf16.h>
@@ -99,56 +99,72 @@ __global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_b
     }
 }
 
-// Rotate-half RoPE in place on the Q and K heads of qkv [B*L, (nq + 2 nkv) * hd], and transpose V into
-// vt [B, nkv, hd, Lp] (keys contiguous) for the P.V product.  cs = [max_seq, hd/2] (cos, sin) table.
-// grid = (ceil(L/32), nq + 2*nkv, B): one CTA per (32 positions, head); 256 threads; 16-byte accesses.
-template <int HD>
-__global__ void __launch_bounds__(256) rope_vt_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ vt,
-                                                      const float2* __restrict__ cs, int L, int Lp, int nq, int nkv) {
+// Split-K tail fused with the next RMSNorm: one CTA per row.
+//   h[row, :]   = bf16( sum over K ranges of partial + residual )          (the projection's output)
+//   out[row, :] = bf16( h * rsqrt(mean(h^2) + eps) * gain )                (h as rounded, like rmsnorm_kernel)
+// N multiple of 8, N/8 <= 8 * blockDim.x.
+__global__ void splitk_reduce_norm_kernel(const float* __restrict__ partial, int split, const __nv_bfloat16* residual,
+                                          __nv_bfloat16* C, int M, int N, const __nv_bfloat16* __restrict__ gain,
+                                          __nv_bfloat16* __restrict__ out, float eps) {
     grid_launch_dependents();
     grid_dependency_wait();
-    constexpr int HALF = HD / 2;
-    constexpr int TPP = HD / 16;                   // threads per position (8 pairs each)
-    const int pos0 = blockIdx.x * 32, head = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
-    const size_t row_stride = (size_t)(nq + 2 * nkv) * HD;
-    if (head < nq + nkv) {
-        const int pl = tid / TPP, j0 = (tid % TPP) * 8, pos = pos0 + pl;
-        if (pl < 32 && pos < L) {
-            __nv_bfloat16* base = qkv + ((size_t)b * L + pos) * row_stride + (size_t)head * HD;
-            uint4 lo = *reinterpret_cast<const uint4*>(base + j0), hi = *reinterpret_cast<const uint4*>(base + HALF + j0);
-            __nv_bfloat16* l8 = reinterpret_cast<__nv_bfloat16*>(&lo);
-            __nv_bfloat16* h8 = reinterpret_cast<__nv_bfloat16*>(&hi);
-            const float2* c = cs + (size_t)pos * HALF + j0;
+    __shared__ float scratch[33];
+    const int row = blockIdx.x, nvec = N / 8;
+    const size_t total = (size_t)M * N, base = (size_t)row * N;
+    constexpr int MAXV = 8;
+    uint4 hbuf[MAXV];
+    float ss = 0.f;
 #pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const float2 k = c[t];
-                const float x0 = __bfloat162float(l8[t]), x1 = __bfloat162float(h8[t]);
-                l8[t] = __float2bfloat16_rn(x0 * k.x - x1 * k.y);
-                h8[t] = __float2bfloat16_rn(x1 * k.x + x0 * k.y);
-            }
-            *reinterpret_cast<uint4*>(base + j0) = lo;
-            *reinterpret_cast<uint4*>(base + HALF + j0) = hi;
-        }
-    } else {
-        __shared__ __align__(16) __nv_bfloat16 tile[32][HD + 8];
-        const int kvh = head - nq - nkv;
-        for (int v = tid; v < 32 * (HD / 8); v += 256) {
-            const int pl = v / (HD / 8), c8 = (v % (HD / 8)) * 8, pos = pos0 + pl;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (pos < L)
-                val = *reinterpret_cast<const uint4*>(qkv + ((size_t)b * L + pos) * row_stride + (size_t)head * HD + c8);
-            *reinterpret_cast<uint4*>(&tile[pl][c8]) = val;
-        }
-        __syncthreads();
-        for (int v = tid; v < HD * 4; v += 256) {
-            const int d = v / 4, g8 = (v % 4) * 8;
-            if (pos0 + g8 < Lp) {
-                uint4 out;
-                __nv_bfloat16* o8 = reinterpret_cast<__nv_bfloat16*>(&out);
+    for (int t = 0; t < MAXV; ++t) {
+        const int i = threadIdx.x + t * blockDim.x;
+        if (i < nvec) {
+            float x[8];
 #pragma unroll
-                for (int t = 0; t < 8; ++t) o8[t] = tile[g8 + t][d];
-                *reinterpret_cast<uint4*>(vt + ((size_t)(b * nkv + kvh) * HD + d) * Lp + pos0 + g8) = out;
+            for (int j = 0; j < 8; ++j) x[j] = 0.f;
+            for (int s = 0; s < split; ++s) {
+                const float4 a = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8);
+                const float4 b = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8 + 4);
+                x[0] += a.x; x[1] += a.y; x[2] += a.z; x[3] += a.w;
+                x[4] += b.x; x[5] += b.y; x[6] += b.z; x[7] += b.w;
             }
+            if (residual) {
+                const uint4 rv = *reinterpret_cast<const uint4*>(residual + base + i * 8);
+                const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 f = __bfloat1622float2(r2[j]);
+                    x[2 * j] += f.x;
+                    x[2 * j + 1] += f.y;
+                }
+            }
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&hbuf[t]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
+                const float2 f = __bfloat1622float2(o2[j]);
+                ss += f.x * f.x + f.y * f.y;
+            }
+            *reinterpret_cast<uint4*>(C + base + i * 8) = hbuf[t];
+        }
+    }
+    ss = block_sum(ss, scratch);
+    const float inv = rsqrtf(ss / (float)N + eps);
+    const uint4* g4 = reinterpret_cast<const uint4*>(gain);
+#pragma unroll
+    for (int t = 0; t < MAXV; ++t) {
+        const int i = threadIdx.x + t * blockDim.x;
+        if (i < nvec) {
+            const uint4 gv = g4[i];
+            uint4 ov;
+            const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&hbuf[t]);
+            const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gv);
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = __bfloat1622float2(b2[j]), g = __bfloat1622float2(g2[j]);
+                o2[j] = __floats2bfloat162_rn(f.x * inv * g.x, f.y * inv * g.y);
+            }
+            *reinterpret_cast<uint4*>(out + base + i * 8) = ov;
         }
     }
 }

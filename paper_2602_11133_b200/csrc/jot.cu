@@ -172,8 +172,17 @@ int pick_split(int M, int N, int K, int sms, size_t scratch_bytes) {
     return split < 1 ? 1 : split;
 }
 
+// An RMSNorm that directly follows a projection; when the projection goes through split-K the norm is
+// folded into the kernel that adds the K ranges (`done` reports whether that happened).
+struct NormAfter {
+    const __nv_bfloat16* gain;
+    __nv_bfloat16* out;
+    float eps;
+    bool done;
+};
+
 int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, int epi, GemmParams p, cudaStream_t st,
-             float* scratch = nullptr, size_t scratch_bytes = 0) {
+             float* scratch = nullptr, size_t scratch_bytes = 0, NormAfter* norm = nullptr) {
     if (epi == EPI_STORE && scratch) {
         const int split = pick_split(p.M, p.N, p.K, di->sms, scratch_bytes);
         if (split > 1) {
@@ -181,6 +190,12 @@ int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, 
             p.partial = scratch;
             const long items = (long)((p.M + 127) / 128) * ((p.N + 255) / 256) * split;
             JOT_TRY((launch_gemm_t<256, EPI_PARTIAL>(p, tmA, w.m256, (int)items, st)));
+            if (norm && p.ldc == p.N && p.N / 8 <= 8 * 256) {
+                launch_k(splitk_reduce_norm_kernel, dim3(p.M), dim3(256), 0, st, scratch, split, p.residual, p.C, p.M, p.N,
+                         norm->gain, norm->out, norm->eps);
+                norm->done = true;
+                return launch_check();
+            }
             const size_t n8 = (size_t)p.M * p.N / 8;
             launch_k(splitk_reduce_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), 0, st, scratch, split, p.residual, p.C, p.M, p.N);
             return launch_check();
@@ -195,6 +210,9 @@ int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, 
     if (epi == EPI_STORE)
         return bn == 256 ? launch_gemm_t<256, EPI_STORE>(p, tmA, w.m256, grid, st)
                          : launch_gemm_t<128, EPI_STORE>(p, tmA, w.m128, grid, st);
+    if (epi == EPI_QKV)
+        return bn == 256 ? launch_gemm_t<256, EPI_QKV>(p, tmA, w.m256, grid, st)
+                         : launch_gemm_t<128, EPI_QKV>(p, tmA, w.m128, grid, st);
     return bn == 256 ? launch_gemm_t<256, EPI_SWIGLU>(p, tmA, w.m256, grid, st)
                      : launch_gemm_t<128, EPI_SWIGLU>(p, tmA, w.m128, grid, st);
 }
@@ -367,25 +385,20 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d);
     }
     JOT_TRY(launch_check());
+    bool norm_ready = false;          // true when a fused split-K tail has already written the next norm into m->a
     for (int l = 0; l < c.n_layers; ++l) {
-        {
+        if (!norm_ready) {
             ProfScope ps(m, JOT_PROF_RMSNORM, st);
             launch_k(rmsnorm_kernel, dim3(M), dim3(256), 0, st, m->h, m->attn_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+            JOT_TRY(launch_check());
         }
-        JOT_TRY(launch_check());
         GemmParams p{};
         p.M = M; p.N = qkv_cols; p.K = d; p.C = m->qkv; p.ldc = qkv_cols; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_QKV, st);
-            JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_STORE, p, st, m->splitk, kSplitKBytes));
+            p.vt = m->vt; p.rope_cs = m->rope_cs; p.L = L; p.Lp = Lp; p.nq = nq; p.nkv = nkv; p.hd = hd;
+            JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_QKV, p, st));
         }
-        {
-            ProfScope ps(m, JOT_PROF_ROPE, st);
-            const dim3 rgrid((L + 31) / 32, nq + 2 * nkv, B);
-            if (hd == 128) launch_k((rope_vt_kernel<128>), dim3(rgrid), dim3(256), 0, st, m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
-            else launch_k((rope_vt_kernel<64>), dim3(rgrid), dim3(256), 0, st, m->qkv, m->vt, m->rope_cs, L, Lp, nq, nkv);
-        }
-        JOT_TRY(launch_check());
         AttnParams ap{};
         ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
         ap.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
@@ -399,13 +412,15 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = d; p.K = nq * hd; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_O, st);
-            JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes));
+            NormAfter na{m->mlp_norm[l], m->a, c.rms_eps, false};
+            JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes, &na));
+            norm_ready = na.done;
         }
-        {
+        if (!norm_ready) {
             ProfScope ps(m, JOT_PROF_RMSNORM, st);
             launch_k(rmsnorm_kernel, dim3(M), dim3(256), 0, st, m->h, m->mlp_norm[l], m->a, d, c.rms_eps, nullptr, nullptr);
+            JOT_TRY(launch_check());
         }
-        JOT_TRY(launch_check());
         p = GemmParams{};
         p.M = M; p.N = 2 * c.d_ff; p.K = d; p.C = m->act; p.ldc = c.d_ff; p.status = status;
         {
@@ -416,7 +431,10 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_DOWN, st);
-            JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st, m->splitk, kSplitKBytes));
+            NormAfter na{l + 1 < c.n_layers ? m->attn_norm[l + 1] : nullptr, m->a, c.rms_eps, false};
+            JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st, m->splitk, kSplitKBytes,
+                             na.gain ? &na : nullptr));
+            norm_ready = na.done;
         }
     }
     return JOT_OK;
