@@ -73,3 +73,47 @@ def bf16_matmul_oracle(a: torch.Tensor, w: torch.Tensor, residual=None) -> torch
     if residual is not None:
         out = out + residual.double()
     return out
+
+
+def replay_trajectory(jot, model, tr: jo.Trajectory, params: jo.JotParams, mask_id: int, ks, bump=None,
+                      from_tolerance=False, rel=REL_TOL):
+    """Teacher-forced replay: every step of the oracle's trajectory is run on the GPU from the oracle's canvas
+    (jot_denoise_step + jot_accept_freeze) and the resulting canvas compared with the oracle's next one.
+
+    A differing position is excused only if the oracle itself says the decision was inside the margin:
+    early-exit test (|r - tau| <= 1e-3 tau), argmax (top-2 gap < 1e-3), or the schedule's pick among
+    candidates whose p1 is within `rel` of the best.  With from_tolerance (models deep or wide enough
+    that the bf16 path's logit noise exceeds 1e-3) the first two margins are the ones the logit tolerance
+    implies: a gap, or |ln r - ln tau|, below 2 * rel * (logit scale).  Returns (steps, excused)."""
+    import torch
+    jp = jot.Params(params.tau_max, params.tau_min, params.gamma, params.D, params.eps)
+    d_bump = dict(bump_id=bump[0].cuda(), bump_val=bump[1].cuda()) if bump is not None else {}
+    excused = 0
+    step_in_block = {}
+    L = len(tr.x)
+    for n, (cv, rep, (lo, hi)) in enumerate(zip(tr.canvases, tr.reports, tr.blocks)):
+        s = step_in_block.get(lo, 0)
+        step_in_block[lo] = s + 1
+        x = torch.tensor([cv], dtype=torch.int32, device="cuda")
+        st = model.denoise_step(x, lo, hi, **d_bump)
+        jot.accept_freeze(jp, mask_id, x, lo, hi, ks[s], st)
+        got = x.cpu()[0].tolist()
+        want = tr.canvases[n + 1] if n + 1 < len(tr.canvases) else tr.x
+        if got == want:
+            continue
+        A = [i for i in range(lo, hi) if cv[i] == mask_id]
+        top1, top2, sumexp = st.top1.cpu()[0], st.top2.cpu()[0], st.sumexp.cpu()[0]
+        p1 = {i: 1.0 / float(sumexp[i]) for i in A}
+        best = max(p1.values())
+        for i in range(L):
+            if got[i] == want[i]:
+                continue
+            scale = max(abs(float(top1[i])), 1.0)
+            margin = 2 * rel * scale if from_tolerance else None
+            near_tau = (i in rep.near_margin) or (
+                margin is not None and abs(math.log(rep.ratio[i]) - math.log(rep.tau[i])) <= margin)
+            near_gap = float(top1[i] - top2[i]) < (margin if margin is not None else GAP_TOL)
+            near_rank = abs(p1.get(i, 0.0) - best) <= rel * best
+            assert near_tau or near_gap or near_rank, (n, i, got[i], want[i], rep.ratio.get(i), rep.tau.get(i))
+            excused += 1
+    return len(tr.canvases), excused
