@@ -75,6 +75,201 @@ __host__ __device__ inline void stats_partition(int R, int grid, int n_vt, int* 
     *n_ch = ch;
 }
 
+// Running LM-head statistics of one output row (EPI_STATS), carried across the vocabulary tiles a CTA visits.
+struct StatsRow {
+    float m1 = -INFINITY, m2 = -INFINITY, S = 0.f;
+    int i1 = 0x7fffffff;
+    int bump_col = -1;
+    float bump_v = 0.f;
+};
+
+// Epilogue of one 128 x BN accumulator tile: the calling thread owns output row `row` (TMEM lane) and reads
+// it 32 columns at a time from tensor memory at `t_acc`.  Shared by the one-CTA and the CTA-pair kernels.
+template <int BN, int EPI>
+__device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_acc, int row, int n_blk, int ks,
+                                              int n_out, StatsRow& st) {
+    constexpr float L2E = 1.4426950408889634f;
+    (void)L2E; (void)ks; (void)n_out; (void)st;
+    if (EPI == EPI_STORE) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            float v[32];
+            tmem_ld32(t_acc + c * 32, v);
+            tmem_ld_wait();
+            const int col0 = n_blk * BN + c * 32;
+            if (row < p.M) {
+                __nv_bfloat16* dst = p.C + (size_t)row * p.ldc + col0;
+                const __nv_bfloat16* res = p.residual ? p.residual + (size_t)row * p.ldc + col0 : nullptr;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    if (col0 + g * 8 < p.N) {         // N is a multiple of 8
+                        float x[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) x[j] = v[g * 8 + j];
+                        if (res) {
+                            uint4 rv = *reinterpret_cast<const uint4*>(res + g * 8);
+                            const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                float2 f = __bfloat1622float2(r2[j]);
+                                x[2 * j] += f.x;
+                                x[2 * j + 1] += f.y;
+                            }
+                        }
+                        uint4 ov;
+                        __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
+                        *reinterpret_cast<uint4*>(dst + g * 8) = ov;
+                    }
+                }
+            }
+        }
+    } else if (EPI == EPI_QKV) {
+        const int hd = p.hd, half = hd >> 1;
+        const int seq = row / p.L, pos = row - seq * p.L;
+#pragma unroll 1
+        for (int hh = 0; hh < BN / hd; ++hh) {
+            const int col_base = n_blk * BN + hh * hd;
+            if (col_base >= p.N) break;
+            const int head = col_base / hd;
+            if (head < p.nq + p.nkv) {
+                // rotate pairs (j, j + hd/2): 32 pairs at a time
+#pragma unroll 1
+                for (int q = 0; q < half / 32; ++q) {
+                    float lo[32], hi[32];
+                    tmem_ld32(t_acc + hh * hd + q * 32, lo);
+                    tmem_ld32(t_acc + hh * hd + half + q * 32, hi);
+                    tmem_ld_wait();
+                    if (row < p.M) {
+                        const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cs + (size_t)pos * half + q * 32);
+                        __nv_bfloat16* dlo = p.C + (size_t)row * p.ldc + col_base + q * 32;
+                        __nv_bfloat16* dhi = dlo + half;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            uint4 olo, ohi;
+                            __nv_bfloat162* l2 = reinterpret_cast<__nv_bfloat162*>(&olo);
+                            __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&ohi);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int e = g * 8 + 2 * j;
+                                const float4 k = cs4[e >> 1];      // (cos, sin) of pairs e and e + 1
+                                // the projection's output is bf16; the rotation acts on the rounded values
+                                const float2 x0 = __bfloat1622float2(__floats2bfloat162_rn(lo[e], lo[e + 1]));
+                                const float2 x1 = __bfloat1622float2(__floats2bfloat162_rn(hi[e], hi[e + 1]));
+                                l2[j] = __floats2bfloat162_rn(x0.x * k.x - x1.x * k.y, x0.y * k.z - x1.y * k.w);
+                                h2[j] = __floats2bfloat162_rn(x1.x * k.x + x0.x * k.y, x1.y * k.z + x0.y * k.w);
+                            }
+                            *reinterpret_cast<uint4*>(dlo + g * 8) = olo;
+                            *reinterpret_cast<uint4*>(dhi + g * 8) = ohi;
+                        }
+                    }
+                }
+            } else {
+                // V head: lane = position, so for a fixed d a warp writes 32 consecutive keys
+                const int kvh = head - p.nq - p.nkv;
+#pragma unroll 1
+                for (int c = 0; c < hd / 32; ++c) {
+                    float v[32];
+                    tmem_ld32(t_acc + hh * hd + c * 32, v);
+                    tmem_ld_wait();
+                    if (row < p.M) {
+                        __nv_bfloat16* dst = p.vt + ((size_t)(seq * p.nkv + kvh) * hd + c * 32) * p.Lp + pos;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) dst[(size_t)j * p.Lp] = __float2bfloat16_rn(v[j]);
+                    }
+                }
+            }
+        }
+    } else if (EPI == EPI_PARTIAL) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            float v[32];
+            tmem_ld32(t_acc + c * 32, v);
+            tmem_ld_wait();
+            const int col0 = n_blk * BN + c * 32;
+            if (row < p.M) {
+                float* dst = p.partial + ((size_t)ks * p.M + row) * p.N + col0;
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                    if (col0 + g * 4 < p.N)           // N is a multiple of 8
+                        *reinterpret_cast<float4*>(dst + g * 4) =
+                            make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+            }
+        }
+    } else if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 64; ++c) {
+            float g[32], u[32];
+            tmem_ld32(t_acc + c * 32, g);
+            tmem_ld32(t_acc + BN / 2 + c * 32, u);
+            tmem_ld_wait();
+            const int col0 = n_blk * (BN / 2) + c * 32;
+            if (row < p.M) {
+                __nv_bfloat16* dst = p.C + (size_t)row * p.ldc + col0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (col0 + q * 8 < n_out) {
+                        uint4 ov;
+                        __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float g0 = g[q * 8 + 2 * j], g1 = g[q * 8 + 2 * j + 1];
+                            float a0 = g0 / (1.f + __expf(-g0)) * u[q * 8 + 2 * j];
+                            float a1 = g1 / (1.f + __expf(-g1)) * u[q * 8 + 2 * j + 1];
+                            o2[j] = __floats2bfloat162_rn(a0, a1);
+                        }
+                        *reinterpret_cast<uint4*>(dst + q * 8) = ov;
+                    }
+                }
+            }
+        }
+    } else {
+        // ---- EPI_STATS: fold this tile's logits into (st.m1, st.i1, st.m2, st.S) ----
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            float v[32];
+            tmem_ld32(t_acc + c * 32, v);
+            tmem_ld_wait();
+            const int col0 = n_blk * BN + c * 32;
+            if (col0 >= p.N) break;                       // whole chunk past the vocabulary
+            unsigned rel_b = (unsigned)(st.bump_col - col0);
+            if (rel_b < 32u) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] += (j == (int)rel_b) ? st.bump_v : 0.f;
+            }
+            unsigned rel_m = (unsigned)(p.mask_col - col0);
+            if (p.mask_col >= 0 && rel_m < 32u) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = (j == (int)rel_m) ? -INFINITY : v[j];
+            }
+            if (col0 + 32 > p.N) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = (col0 + j < p.N) ? v[j] : -INFINITY;
+            }
+            float cm = v[0];
+#pragma unroll
+            for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+            const float old_m = st.m1;
+            if (cm > st.m2) {                                // only then can the top two change
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float x = v[j];
+                    st.m2 = fmaxf(st.m2, fminf(x, st.m1));         // runner-up as an order statistic
+                    st.i1 = (x > st.m1) ? col0 + j : st.i1;        // strict: the lowest index wins ties
+                    st.m1 = fmaxf(st.m1, x);
+                }
+            }
+            // st.S = sum exp(l - st.m1): rescale what was summed against the old maximum
+            const float nm = st.m1 * L2E;
+            float acc_s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(v[j], L2E, -nm));
+            st.S = st.S * ex2_approx(old_m * L2E - nm) + acc_s;
+        }
+    }
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB) {
@@ -228,208 +423,21 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         int acc = 0;
         uint32_t acc_phase = 0;
         int m_blk, n_blk;
-
-        // EPI_STATS running state of this thread's row
-        float m1 = -INFINITY, m2 = -INFINITY, S = 0.f;
-        int i1 = 0x7fffffff;
-        int bump_col = -1;
-        float bump_v = 0.f;
-        constexpr float L2E = 1.4426950408889634f;
+        StatsRow st;
         if (EPI == EPI_STATS && total_tiles > 0) {
             int R = *p.d_R;
             int row = m_blk0 * kBM + row_in_tile;
             if (row < R && p.bump_id != nullptr) {
                 int flat = p.rows[row];
-                bump_col = p.bump_id[flat];
-                bump_v = p.bump_val[flat];
+                st.bump_col = p.bump_id[flat];
+                st.bump_v = p.bump_val[flat];
             }
         }
-
         bool ok = true;
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t t_acc = lane_base + acc * BN;
-            const int row = m_blk * kBM + row_in_tile;
-
-            if (EPI == EPI_STORE) {
-#pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    float v[32];
-                    tmem_ld32(t_acc + c * 32, v);
-                    tmem_ld_wait();
-                    const int col0 = n_blk * BN + c * 32;
-                    if (row < p.M) {
-                        __nv_bfloat16* dst = p.C + (size_t)row * p.ldc + col0;
-                        const __nv_bfloat16* res = p.residual ? p.residual + (size_t)row * p.ldc + col0 : nullptr;
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            if (col0 + g * 8 < p.N) {         // N is a multiple of 8
-                                float x[8];
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) x[j] = v[g * 8 + j];
-                                if (res) {
-                                    uint4 rv = *reinterpret_cast<const uint4*>(res + g * 8);
-                                    const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
-#pragma unroll
-                                    for (int j = 0; j < 4; ++j) {
-                                        float2 f = __bfloat1622float2(r2[j]);
-                                        x[2 * j] += f.x;
-                                        x[2 * j + 1] += f.y;
-                                    }
-                                }
-                                uint4 ov;
-                                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
-                                *reinterpret_cast<uint4*>(dst + g * 8) = ov;
-                            }
-                        }
-                    }
-                }
-            } else if (EPI == EPI_QKV) {
-                const int hd = p.hd, half = hd >> 1;
-                const int seq = row / p.L, pos = row - seq * p.L;
-#pragma unroll 1
-                for (int hh = 0; hh < BN / hd; ++hh) {
-                    const int col_base = n_blk * BN + hh * hd;
-                    if (col_base >= p.N) break;
-                    const int head = col_base / hd;
-                    if (head < p.nq + p.nkv) {
-                        // rotate pairs (j, j + hd/2): 32 pairs at a time
-#pragma unroll 1
-                        for (int q = 0; q < half / 32; ++q) {
-                            float lo[32], hi[32];
-                            tmem_ld32(t_acc + hh * hd + q * 32, lo);
-                            tmem_ld32(t_acc + hh * hd + half + q * 32, hi);
-                            tmem_ld_wait();
-                            if (row < p.M) {
-                                const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cs + (size_t)pos * half + q * 32);
-                                __nv_bfloat16* dlo = p.C + (size_t)row * p.ldc + col_base + q * 32;
-                                __nv_bfloat16* dhi = dlo + half;
-#pragma unroll
-                                for (int g = 0; g < 4; ++g) {
-                                    uint4 olo, ohi;
-                                    __nv_bfloat162* l2 = reinterpret_cast<__nv_bfloat162*>(&olo);
-                                    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&ohi);
-#pragma unroll
-                                    for (int j = 0; j < 4; ++j) {
-                                        const int e = g * 8 + 2 * j;
-                                        const float4 k = cs4[e >> 1];      // (cos, sin) of pairs e and e + 1
-                                        // the projection's output is bf16; the rotation acts on the rounded values
-                                        const float2 x0 = __bfloat1622float2(__floats2bfloat162_rn(lo[e], lo[e + 1]));
-                                        const float2 x1 = __bfloat1622float2(__floats2bfloat162_rn(hi[e], hi[e + 1]));
-                                        l2[j] = __floats2bfloat162_rn(x0.x * k.x - x1.x * k.y, x0.y * k.z - x1.y * k.w);
-                                        h2[j] = __floats2bfloat162_rn(x1.x * k.x + x0.x * k.y, x1.y * k.z + x0.y * k.w);
-                                    }
-                                    *reinterpret_cast<uint4*>(dlo + g * 8) = olo;
-                                    *reinterpret_cast<uint4*>(dhi + g * 8) = ohi;
-                                }
-                            }
-                        }
-                    } else {
-                        // V head: lane = position, so for a fixed d a warp writes 32 consecutive keys
-                        const int kvh = head - p.nq - p.nkv;
-#pragma unroll 1
-                        for (int c = 0; c < hd / 32; ++c) {
-                            float v[32];
-                            tmem_ld32(t_acc + hh * hd + c * 32, v);
-                            tmem_ld_wait();
-                            if (row < p.M) {
-                                __nv_bfloat16* dst = p.vt + ((size_t)(seq * p.nkv + kvh) * hd + c * 32) * p.Lp + pos;
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) dst[(size_t)j * p.Lp] = __float2bfloat16_rn(v[j]);
-                            }
-                        }
-                    }
-                }
-            } else if (EPI == EPI_PARTIAL) {
-#pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    float v[32];
-                    tmem_ld32(t_acc + c * 32, v);
-                    tmem_ld_wait();
-                    const int col0 = n_blk * BN + c * 32;
-                    if (row < p.M) {
-                        float* dst = p.partial + ((size_t)ks * p.M + row) * p.N + col0;
-#pragma unroll
-                        for (int g = 0; g < 8; ++g)
-                            if (col0 + g * 4 < p.N)           // N is a multiple of 8
-                                *reinterpret_cast<float4*>(dst + g * 4) =
-                                    make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
-                    }
-                }
-            } else if (EPI == EPI_SWIGLU) {
-#pragma unroll 1
-                for (int c = 0; c < BN / 64; ++c) {
-                    float g[32], u[32];
-                    tmem_ld32(t_acc + c * 32, g);
-                    tmem_ld32(t_acc + BN / 2 + c * 32, u);
-                    tmem_ld_wait();
-                    const int col0 = n_blk * (BN / 2) + c * 32;
-                    if (row < p.M) {
-                        __nv_bfloat16* dst = p.C + (size_t)row * p.ldc + col0;
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            if (col0 + q * 8 < n_out) {
-                                uint4 ov;
-                                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    float g0 = g[q * 8 + 2 * j], g1 = g[q * 8 + 2 * j + 1];
-                                    float a0 = g0 / (1.f + __expf(-g0)) * u[q * 8 + 2 * j];
-                                    float a1 = g1 / (1.f + __expf(-g1)) * u[q * 8 + 2 * j + 1];
-                                    o2[j] = __floats2bfloat162_rn(a0, a1);
-                                }
-                                *reinterpret_cast<uint4*>(dst + q * 8) = ov;
-                            }
-                        }
-                    }
-                }
-            } else {
-                // ---- EPI_STATS: fold this tile's logits into (m1, i1, m2, S) ----
-#pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    float v[32];
-                    tmem_ld32(t_acc + c * 32, v);
-                    tmem_ld_wait();
-                    const int col0 = n_blk * BN + c * 32;
-                    if (col0 >= p.N) break;                       // whole chunk past the vocabulary
-                    unsigned rel_b = (unsigned)(bump_col - col0);
-                    if (rel_b < 32u) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] += (j == (int)rel_b) ? bump_v : 0.f;
-                    }
-                    unsigned rel_m = (unsigned)(p.mask_col - col0);
-                    if (p.mask_col >= 0 && rel_m < 32u) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = (j == (int)rel_m) ? -INFINITY : v[j];
-                    }
-                    if (col0 + 32 > p.N) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = (col0 + j < p.N) ? v[j] : -INFINITY;
-                    }
-                    float cm = v[0];
-#pragma unroll
-                    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
-                    const float old_m = m1;
-                    if (cm > m2) {                                // only then can the top two change
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            float x = v[j];
-                            m2 = fmaxf(m2, fminf(x, m1));         // runner-up as an order statistic
-                            i1 = (x > m1) ? col0 + j : i1;        // strict: the lowest index wins ties
-                            m1 = fmaxf(m1, x);
-                        }
-                    }
-                    // S = sum exp(l - m1): rescale what was summed against the old maximum
-                    const float nm = m1 * L2E;
-                    float acc_s = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(v[j], L2E, -nm));
-                    S = S * ex2_approx(old_m * L2E - nm) + acc_s;
-                }
-            }
+            epilogue_tile<BN, EPI>(p, lane_base + acc * BN, m_blk * kBM + row_in_tile, n_blk, ks, n_out, st);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
@@ -438,7 +446,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         }
         if (EPI == EPI_STATS && ok && total_tiles > 0) {
             p.partials[(size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile] =
-                make_float4(m1, __int_as_float(i1), m2, S);
+                make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
         }
     }
 
