@@ -1,0 +1,209 @@
+// CTA-pair variant of the projection kernel (tcgen05 cta_group::2): two CTAs of a cluster share one
+// 256 x 256 output tile.  Each CTA loads its own 128 rows of A and its own half (128 rows) of the W tile,
+// the even-ranked CTA issues UMMA 256 x 256 x 16 for both, and each CTA's tensor memory receives its
+// 128 rows x 256 columns, which its own epilogue warps drain.  Per CTA and k-block that is 32 KB of
+// operands for the same 4.2 MFLOP that cost the one-CTA kernel 48 KB, which is what the shared-memory
+// ingest of an SM limits.  Epilogues are those of gemm.cuh (store, SwiGLU, QKV + RoPE, LM-head statistics).
+//
+// Barriers (same shared-memory offsets in both CTAs):
+//   full[s]      leader's only: 1 arrival (leader's expect_tx for both CTAs' bytes) + bytes of both CTAs' loads
+//   empty[s]     each CTA's own: arrives through the leader's commit, delivered to both CTAs
+//   acc_full[a]  each CTA's own: same mechanism
+//   acc_empty[a] leader's only: 8 arrivals = 4 epilogue warps x 2 CTAs (the peer arrives remotely)
+#pragma once
+#include "gemm.cuh"
+
+namespace jot {
+
+constexpr int kPairStages = 6;
+constexpr int kPairStageBytes = 2 * kBM * kBK * 2;                 // A tile + half W tile per CTA
+constexpr int kPairDynBytes = kPairStages * kPairStageBytes + 1024;
+
+// Row-block pairs and vocabulary chunks of the pair kernel's LM-head schedule.
+__host__ __device__ inline void stats_partition_pair(int R, int n_clusters, int n_vt, int* n_rb, int* n_pr, int* n_ch) {
+    const int rb = (R + kBM - 1) / kBM, pr = (rb + 1) / 2;
+    int ch = pr > 0 ? n_clusters / pr : 0;
+    if (ch > n_vt) ch = n_vt;
+    *n_rb = rb;
+    *n_pr = pr;
+    *n_ch = ch;
+}
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB) {
+    constexpr int BN = 256, STAGES = kPairStages;
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t IDESC = umma_idesc_bf16(256, BN);
+    constexpr int HALF_BYTES = kBM * kBK * 2;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = (int)cluster_ctarank();
+    const bool leader = rank == 0;
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    const int num_kb = (p.K + kBK - 1) / kBK;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 8);
+        }
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(&tmem_base_slot, TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    cluster_sync_all();                       // both CTAs' barriers exist before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    grid_launch_dependents();
+    grid_dependency_wait();
+
+    // ---- schedule: pair tiles (two row blocks x one 256-wide column block), identical in every role ----
+    const int num_m = (p.M + kBM - 1) / kBM, num_pm = (num_m + 1) / 2;
+    constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
+    const int n_out = (EPI == EPI_SWIGLU) ? p.N / 2 : p.N;
+    const int num_n = (n_out + BN_OUT - 1) / BN_OUT;
+    int total_tiles = num_pm * num_n;
+    int m_blk0 = 0, n_first = 0, chunk = 0;
+    bool stats_row_block_valid = false;
+    if (EPI == EPI_STATS) {
+        int n_rb, n_pr, n_ch;
+        stats_partition_pair(*p.d_R, n_clusters, num_n, &n_rb, &n_pr, &n_ch);
+        chunk = n_pr > 0 ? cluster_id / n_pr : 0;
+        total_tiles = 0;
+        if (n_pr > 0 && chunk < n_ch) {
+            m_blk0 = 2 * (cluster_id % n_pr) + rank;
+            stats_row_block_valid = m_blk0 < n_rb;
+            n_first = (int)((long long)chunk * num_n / n_ch);
+            total_tiles = (int)((long long)(chunk + 1) * num_n / n_ch) - n_first;
+        }
+    }
+    auto tile_at = [&](int it, int& m_blk, int& n_blk) -> bool {
+        if (EPI == EPI_STATS) {
+            if (it >= total_tiles) return false;
+            m_blk = m_blk0;
+            n_blk = n_first + it;
+            return true;
+        }
+        const int t = cluster_id + it * n_clusters;
+        if (t >= total_tiles) return false;
+        m_blk = 2 * (t % num_pm) + rank;          // row-block pairs fastest: neighbours share the W tile
+        n_blk = t / num_pm;
+        return true;
+    };
+
+    if (warp == 0) {
+        // ================= TMA producer (both CTAs) =================
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int m_blk, n_blk;
+            bool ok = true;
+            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+                // this CTA's half of the W tile: SwiGLU pairs 128 gate rows (leader) with the matching 128 up rows
+                const int w_row = (EPI == EPI_SWIGLU) ? (rank == 0 ? n_blk * kBM : p.N / 2 + n_blk * kBM)
+                                                      : n_blk * BN + rank * kBM;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
+                    uint8_t* sA = smem + stage * kPairStageBytes;
+                    uint8_t* sB = sA + HALF_BYTES;
+                    const uint32_t full_leader = mapa_u32(&full_bar[stage], 0);
+                    if (leader) mbar_arrive_expect_tx(&full_bar[stage], 2 * kPairStageBytes);
+                    tma_load_2d_pair(sA, &tmA, full_leader, kb * kBK, m_blk * kBM);
+                    tma_load_2d_pair(sB, &tmB, full_leader, kb * kBK, w_row);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer (leader CTA only) =================
+        if (lane == 0 && leader) {
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            int m_blk, n_blk;
+            bool ok = true;
+            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abortp)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + stage * kPairStageBytes);
+                    const uint32_t b_addr = a_addr + HALF_BYTES;
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        umma_bf16_pair(d_tmem, umma_desc_k128(a_addr + k * 32), umma_desc_k128(b_addr + k * 32), IDESC,
+                                       (kb | k) != 0);
+                    }
+                    umma_commit_pair(&empty_bar[stage], 0x3);     // both CTAs may refill this stage
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit_pair(&acc_full[acc], 0x3);            // both CTAs' accumulators are complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ================= epilogue (warps 2..5, both CTAs) =================
+        const int quad = warp & 3;
+        const int row_in_tile = quad * 32 + lane;
+        const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        int m_blk, n_blk;
+        StatsRow st;
+        if (EPI == EPI_STATS && total_tiles > 0) {
+            const int row = m_blk0 * kBM + row_in_tile;
+            if (row < *p.d_R && p.bump_id != nullptr) {
+                const int flat = p.rows[row];
+                st.bump_col = p.bump_id[flat];
+                st.bump_v = p.bump_val[flat];
+            }
+        }
+        bool ok = true;
+        for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+            if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
+            tc_fence_after();
+            epilogue_tile<BN, EPI>(p, lane_base + acc * BN, m_blk * kBM + row_in_tile, n_blk, 0, n_out, st);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_u32(&acc_empty[acc], 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+        if (EPI == EPI_STATS && ok && total_tiles > 0 && stats_row_block_valid) {
+            p.partials[(size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile] =
+                make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
+        }
+    }
+
+    // ---- teardown: nobody leaves while the other CTA may still signal or read across ----
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+    if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, 3);
+}
+
+}  // namespace jot

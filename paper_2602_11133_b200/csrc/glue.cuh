@@ -230,7 +230,7 @@ __device__ __forceinline__ StatTuple merge_tuples(const StatTuple& a, const Stat
     return r;
 }
 __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restrict__ partials, int R_pad, int grid_gemm,
-                                                          int n_vt, const int32_t* __restrict__ rows,
+                                                          int n_vt, int pair_mode, const int32_t* __restrict__ rows,
                                                           const int32_t* __restrict__ d_R, float* __restrict__ top1,
                                                           float* __restrict__ top2, float* __restrict__ sumexp,
                                                           int32_t* __restrict__ argmax) {
@@ -239,8 +239,9 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
     const int R = *d_R;
     const int r = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= R) return;
+    // the same split of the vocabulary into chunks as the kernel that wrote the partial tuples
     const int n_rb = (R + 127) / 128;
-    int n_ch = grid_gemm / n_rb;
+    int n_ch = pair_mode ? (grid_gemm / 2) / ((n_rb + 1) / 2) : grid_gemm / n_rb;
     if (n_ch > n_vt) n_ch = n_vt;
     StatTuple t{-INFINITY, -INFINITY, 0.f, 0x7fffffff};
     for (int c = lane; c < n_ch; c += 32) {

@@ -16,6 +16,7 @@
 #include "accept.cuh"
 #include "attention.cuh"
 #include "gemm.cuh"
+#include "gemm2.cuh"
 #include "glue.cuh"
 
 using namespace jot;
@@ -142,12 +143,30 @@ int launch_gemm_t(const GemmParams& p, const CUtensorMap& tmA, const CUtensorMap
     return launch_check();
 }
 
-// Tile width for a plain projection: the one that needs the least (waves x tile width).
-int pick_bn(int M, int n_out, int sms) {
-    long m_blks = (M + 127) / 128;
-    long t256 = m_blks * ((n_out + 255) / 256), t128 = m_blks * ((n_out + 127) / 128);
-    long c256 = ((t256 + sms - 1) / sms) * 256, c128 = ((t128 + sms - 1) / sms) * 128;
-    return c128 < c256 ? 128 : 256;
+template <int EPI>
+int launch_pair_t(const GemmParams& p, const CUtensorMap& tmA, const CUtensorMap& tmB, int grid, cudaStream_t st) {
+    static thread_local bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev & 63]) {
+        JOT_CUDA(cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairDynBytes));
+        attr_set[dev & 63] = true;
+    }
+    launch_k((gemm_pair_kernel<EPI>), dim3(grid & ~1), dim3(kGemmThreads), kPairDynBytes, st, p, tmA, tmB);
+    return launch_check();
+}
+
+// Which kernel shape moves the fewest operand bytes through an SM for this projection: waves x bytes per
+// k-block (48 KB for a 128 x 256 tile, 32 KB for a 128 x 128 tile, 32 KB per CTA of a 256 x 256 pair tile).
+enum { SHAPE_256 = 0, SHAPE_128 = 1, SHAPE_PAIR = 2 };
+int pick_shape(int M, int n_out, int sms, bool allow_128) {
+    const long m_blks = (M + 127) / 128, n256 = (n_out + 255) / 256, n128 = (n_out + 127) / 128;
+    auto waves = [](long tiles, long slots) { return (tiles + slots - 1) / slots; };
+    const long c256 = waves(m_blks * n256, sms) * 48;
+    const long c128 = allow_128 ? waves(m_blks * n128, sms) * 32 : (1L << 60);
+    const long cpair = m_blks >= 2 ? waves(((m_blks + 1) / 2) * n256, sms / 2) * 32 : (1L << 60);
+    if (c256 <= c128 && c256 <= cpair) return SHAPE_256;
+    return cpair <= c128 ? SHAPE_PAIR : SHAPE_128;
 }
 
 struct WeightMaps {     // one weight matrix as B operand, for both tile widths
@@ -201,8 +220,19 @@ int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, 
             return launch_check();
         }
     }
+    // for SwiGLU a "256-wide" tile holds 128 gate + 128 up columns, i.e. 128 output columns
     const int n_out = (epi == EPI_SWIGLU) ? p.N / 2 : p.N;
-    int bn = pick_bn(p.M, epi == EPI_SWIGLU ? 2 * n_out : n_out, di->sms);
+    const int n_eff = (epi == EPI_SWIGLU) ? 2 * n_out : n_out;
+    const int shape = pick_shape(p.M, n_eff, di->sms, true);
+    if (shape == SHAPE_PAIR) {
+        const long tiles = (long)(((p.M + 127) / 128 + 1) / 2) * ((n_eff + 255) / 256);
+        const int grid = (int)(2 * tiles < di->sms ? 2 * tiles : di->sms);
+        // each CTA of a pair fetches 128 rows of W: the 128-row box of the plain maps, the 128-row box of SwiGLU's
+        if (epi == EPI_STORE) return launch_pair_t<EPI_STORE>(p, tmA, w.m128, grid, st);
+        if (epi == EPI_QKV) return launch_pair_t<EPI_QKV>(p, tmA, w.m128, grid, st);
+        return launch_pair_t<EPI_SWIGLU>(p, tmA, w.m256, grid, st);
+    }
+    const int bn = shape == SHAPE_128 ? 128 : 256;
     const int bn_out = (epi == EPI_SWIGLU) ? bn / 2 : bn;
     long tiles = (long)((p.M + 127) / 128) * ((n_out + bn_out - 1) / bn_out);
     int grid = (int)(tiles < di->sms ? tiles : di->sms);
@@ -449,18 +479,27 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     p.d_R = m->ctrl + 1; p.rows = m->rows; p.bump_id = bump_id; p.bump_val = bump_val;
     p.mask_col = exclude_mask ? c.mask_id : -1;
     p.partials = m->partials; p.R_pad = m->R_cap;
-    const int grid = m->di->sms > 256 ? 256 : m->di->sms;
-    // few active rows: the head streams W once and is bandwidth bound -> narrower tiles balance the SMs better
-    const int bn = (M <= 256) ? 128 : 256;
+    // few active rows: the head streams W once and is bandwidth bound -> narrow tiles balance the SMs best;
+    // many rows: CTA pairs (256 x 256 tiles) halve the W bytes each SM takes in
+    const int mode = (M <= 128) ? 0 : (M <= 256 ? 1 : 2);
+    int grid = m->di->sms > 256 ? 256 : m->di->sms;
+    int bn = 256;
     {
         ProfScope ps(m, JOT_PROF_LM_HEAD, st);
-        if (bn == 256) JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
-        else JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+        if (mode == 0) {
+            bn = 128;
+            JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+        } else if (mode == 1) {
+            JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
+        } else {
+            grid &= ~1;
+            JOT_TRY((launch_pair_t<EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+        }
     }
     const int n_vt = (c.vocab + bn - 1) / bn;
     ProfScope ps(m, JOT_PROF_MERGE, st);
-    launch_k(merge_stats_kernel, dim3((M + 3) / 4), dim3(128), 0, st, m->partials, m->R_cap, grid, n_vt, m->rows, m->ctrl + 1,
-                                                               top1, top2, sumexp, argmax);
+    launch_k(merge_stats_kernel, dim3((M + 3) / 4), dim3(128), 0, st, m->partials, m->R_cap, grid, n_vt, mode == 2 ? 1 : 0,
+             m->rows, m->ctrl + 1, top1, top2, sumexp, argmax);
     return launch_check();
 }
 

@@ -25,6 +25,7 @@ def jot():
 @pytest.mark.parametrize("M,N,K", [
     (128, 256, 64), (96, 768, 256), (96, 256, 704), (384, 4096, 4096), (200, 1408, 256),
     (384, 12288, 4096), (1000, 3584, 1024), (130, 136, 72),
+    (1024, 4096, 1024), (640, 1024, 512), (2048, 8192, 512), (300, 520, 200),      # CTA-pair tiles, odd row-block counts
 ])
 @pytest.mark.parametrize("with_res", [False, True])
 def test_gemm_matches_float64_definition(jot, M, N, K, with_res):
