@@ -430,9 +430,10 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
             JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_QKV, p, st));
         }
         AttnParams ap{};
-        ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
+        ap.B = B; ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
         ap.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
-        dim3 grid((L + 127) / 128, nq, B);
+        const long items = (long)B * nq * ((L + 127) / 128);
+        dim3 grid((unsigned)(items < m->di->sms ? items : m->di->sms));
         {
             ProfScope ps(m, JOT_PROF_ATTENTION, st);
             if (hd == 128) JOT_TRY(launch_attention_t<128>(ap, m->tm_qkv3, m->tm_vt, grid, st));
