@@ -85,10 +85,13 @@ typedef struct {
 /* Generation settings of Algorithm 1.  gen_len = number of masked positions appended to the prompt;
  * steps = T; block_len = semi-autoregressive block size (gen_len for a single block; must divide
  * gen_len, and gen_len/block_len must divide steps).  exclude_mask_token != 0 keeps the mask token
- * out of the candidate predictions. */
+ * out of the candidate predictions.  compact_finished: the paper decodes one sequence at a time, where
+ * early stopping ends the loop; in a batch the loop runs until the slowest sequence is done, and with this
+ * flag the forward pass only covers the sequences still decoding (same tokens and step counts, fewer rows). */
 typedef struct {
     int32_t gen_len, steps, block_len;
     int32_t exclude_mask_token;
+    int32_t compact_finished;   /* != 0: sequences that have finished drop out of later forward passes */
 } jot_gen_config;
 
 typedef struct jot_model jot_model; /* opaque; host-side object owned by the library */

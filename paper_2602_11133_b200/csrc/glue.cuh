@@ -33,13 +33,16 @@ __device__ __forceinline__ float block_sum(float v, float* scratch /* >= 33 floa
     return r;
 }
 
-// h[row, :] = E[tokens[row], :]          one CTA per row, 16-byte copies (d multiple of 8)
+// h[row, :] = E[token of that row, :]     one CTA per row, 16-byte copies (d multiple of 8).
+// With seq_map the rows are those of a compacted batch: row = (b', i) reads tokens[seq_map[b'], i].
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E,
-                             __nv_bfloat16* __restrict__ h, int d) {
+                             __nv_bfloat16* __restrict__ h, int d, int L, const int32_t* __restrict__ seq_map) {
     grid_launch_dependents();
     grid_dependency_wait();
     const int row = blockIdx.x;
-    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[row] * d);
+    int src_row = row;
+    if (seq_map) src_row = seq_map[row / L] * L + row % L;
+    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[src_row] * d);
     uint4* dst = reinterpret_cast<uint4*>(h + (size_t)row * d);
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = src[i];
 }
@@ -170,11 +173,15 @@ __global__ void splitk_reduce_norm_kernel(const float* __restrict__ partial, int
 }
 
 // Active rows of the step: every position of [lo_b, hi_b) that holds mask_id, in (b, i) order.
-// Single CTA.  rows[r] = b*L + i; *d_R = count.  With `state`, each sequence uses its own block.
+// Single CTA.  rows_out[r] = b*L + i (index into the caller's [B, L] arrays); rows[r] = the same row's index
+// in the forward pass's activation matrix, which differs when finished sequences were compacted away
+// (seq_map: compact slot -> sequence; n_seq slots).  *d_R = count.  With `state`, each sequence uses its
+// own block and finished sequences contribute nothing.
 __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restrict__ tokens, int B, int L,
                                                           int32_t mask_id, int blk_lo, int blk_hi,
                                                           const SeqState* __restrict__ state, int P, int block_len,
-                                                          int n_blocks, int32_t* __restrict__ rows,
+                                                          int n_blocks, const int32_t* __restrict__ seq_map,
+                                                          int32_t* __restrict__ rows, int32_t* __restrict__ rows_out,
                                                           int32_t* __restrict__ d_R) {
     grid_launch_dependents();
     grid_dependency_wait();
@@ -183,7 +190,8 @@ __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restr
     const int tid = threadIdx.x, wid = tid >> 5, ln = tid & 31;
     if (tid == 0) total = 0;
     __syncthreads();
-    for (int b = 0; b < B; ++b) {
+    for (int slot = 0; slot < B; ++slot) {
+        const int b = seq_map ? seq_map[slot] : slot;
         int lo = blk_lo, hi = blk_hi;
         if (state) {
             const int blk = state[b].blk;
@@ -199,7 +207,11 @@ __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restr
             __syncthreads();
             int off = total;
             for (int w = 0; w < wid; ++w) off += warp_counts[w];
-            if (c) rows[off + __popc(bal & ((1u << ln) - 1u))] = b * L + i;
+            if (c) {
+                const int r = off + __popc(bal & ((1u << ln) - 1u));
+                rows[r] = slot * L + i;
+                rows_out[r] = b * L + i;
+            }
             __syncthreads();
             if (tid == 0) {
                 int t = 0;
@@ -264,6 +276,23 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
         sumexp[flat] = t.S;
         argmax[flat] = t.i1;
     }
+}
+
+// Sequences that still have work, in ascending order: seq_map[slot] = b, *n_active = count.  One warp.
+__global__ void build_seq_map_kernel(const SeqState* __restrict__ state, int B, int n_blocks,
+                                     int32_t* __restrict__ seq_map, int32_t* __restrict__ n_active) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int ln = threadIdx.x;
+    int total = 0;
+    for (int base = 0; base < B; base += 32) {
+        const int b = base + ln;
+        const bool live = b < B && state[b].blk < n_blocks;
+        const uint32_t bal = __ballot_sync(0xffffffffu, live);
+        if (live) seq_map[total + __popc(bal & ((1u << ln) - 1u))] = b;
+        total += __popc(bal);
+    }
+    if (ln == 0) *n_active = total;
 }
 
 // x = [prompt ; mask_id * G]  and fresh loop state  (Algorithm 1, initialisation)

@@ -279,7 +279,7 @@ struct jot_model {
     int32_t* ctrl;        // [0] status, [1] R, [2] n_unfinished
     float2* rope_cs;
     __nv_bfloat16 *h, *a, *qkv, *vt, *attn, *act, *hsel;
-    int32_t* rows;
+    int32_t *rows, *rows_out, *seq_map;
     float4* partials;
     float* splitk;
     int R_cap;
@@ -333,7 +333,7 @@ struct ProfScope {
 };
 
 struct Layout {
-    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, partials, splitk, canvas, top1, top2, sumexp, argmax, state, params,
+    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, rows_out, seq_map, partials, splitk, canvas, top1, top2, sumexp, argmax, state, params,
         total;
 };
 
@@ -371,6 +371,8 @@ Layout make_layout(const jot_model_config* c, int max_batch, int max_seq) {
     l.act = take(M * (size_t)c->d_ff * 2);
     l.hsel = take(R_cap * c->d_model * 2);
     l.rows = take(R_cap * 4);
+    l.rows_out = take(R_cap * 4);
+    l.seq_map = take((size_t)max_batch * 4);
     l.partials = take((size_t)256 * R_cap * sizeof(float4));   // up to 256 vocabulary chunks
     l.splitk = take(kSplitKBytes);
     l.canvas = take(M * 4);
@@ -402,7 +404,8 @@ int encode_activation_maps(jot_model* m, int B, int L) {
 }
 
 // Transformer body: tokens [B, L] -> residual stream m->h [B*L, d] (before the final norm).
-int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream_t st) {
+// B sequences are processed; with seq_map they are the compacted batch (slot -> sequence of d_tokens).
+int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream_t st, const int32_t* seq_map = nullptr) {
     const jot_model_config& c = m->cfg;
     const int M = B * L, d = c.d_model, hd = c.head_dim, nq = c.n_q_heads, nkv = c.n_kv_heads;
     const int qkv_cols = (nq + 2 * nkv) * hd;
@@ -412,7 +415,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
 
     {
         ProfScope ps(m, JOT_PROF_EMBED, st);
-        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d);
+        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d, L, seq_map);
     }
     JOT_TRY(launch_check());
     bool norm_ready = false;          // true when a fused split-K tail has already written the next norm into m->a
@@ -477,7 +480,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     const jot_model_config& c = m->cfg;
     GemmParams p{};
     p.M = m->R_cap; p.N = c.vocab; p.K = c.d_model; p.status = m->ctrl;
-    p.d_R = m->ctrl + 1; p.rows = m->rows; p.bump_id = bump_id; p.bump_val = bump_val;
+    p.d_R = m->ctrl + 1; p.rows = m->rows_out; p.bump_id = bump_id; p.bump_val = bump_val;
     p.mask_col = exclude_mask ? c.mask_id : -1;
     p.partials = m->partials; p.R_pad = m->R_cap;
     // few active rows: the head streams W once and is bandwidth bound -> narrow tiles balance the SMs best;
@@ -500,7 +503,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     const int n_vt = (c.vocab + bn - 1) / bn;
     ProfScope ps(m, JOT_PROF_MERGE, st);
     launch_k(merge_stats_kernel, dim3((M + 3) / 4), dim3(128), 0, st, m->partials, m->R_cap, grid, n_vt, mode == 2 ? 1 : 0,
-             m->rows, m->ctrl + 1, top1, top2, sumexp, argmax);
+             m->rows_out, m->ctrl + 1, top1, top2, sumexp, argmax);
     return launch_check();
 }
 
@@ -604,6 +607,8 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
     m->act = (__nv_bfloat16*)(base + lay.act);
     m->hsel = (__nv_bfloat16*)(base + lay.hsel);
     m->rows = (int32_t*)(base + lay.rows);
+    m->rows_out = (int32_t*)(base + lay.rows_out);
+    m->seq_map = (int32_t*)(base + lay.seq_map);
     m->partials = (float4*)(base + lay.partials);
     m->splitk = (float*)(base + lay.splitk);
     m->R_cap = (int)align_up((size_t)max_batch * max_seq, 128);
@@ -650,6 +655,7 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
     if (e == cudaSuccess) e = cudaMemset(m->ctrl, 0, 1024);
     if (e == cudaSuccess) e = cudaMemset(m->hsel, 0, (size_t)m->R_cap * d * 2);
     if (e == cudaSuccess) e = cudaMemset(m->rows, 0, (size_t)m->R_cap * 4);
+    if (e == cudaSuccess) e = cudaMemset(m->rows_out, 0, (size_t)m->R_cap * 4);
     if (e == cudaSuccess) e = cudaHostAlloc((void**)&m->h_pinned, 64 + (size_t)max_batch * sizeof(SeqState), cudaHostAllocDefault);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
@@ -676,7 +682,7 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
     JOT_TRY(encode_activation_maps(m, B, L));
     {
         ProfScope ps(m, JOT_PROF_ROWS, st);
-        launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+        launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, nullptr, m->rows, m->rows_out,
                                               m->ctrl + 1);
         JOT_TRY(launch_check());
         launch_k(gather_rows_kernel, dim3(B * L), dim3(128), 0, st, (const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
@@ -696,7 +702,7 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
     JOT_TRY(forward_body(m, d_tokens, B, L, st));
     {
         ProfScope ps(m, JOT_PROF_ROWS, st);
-        launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, m->rows,
+        launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, nullptr, m->rows, m->rows_out,
                                               m->ctrl + 1);
         JOT_TRY(launch_check());
         launch_k(rmsnorm_kernel, dim3(B * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
@@ -752,20 +758,30 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
                                                            m->state);
     JOT_TRY(launch_check());
     int passes = 0;
+    int B_act = B;                                   // sequences that still have work (known from the last step)
+    const bool compact = gen->compact_finished != 0;
     for (int it = 0; it < gen->steps; ++it) {
         JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
-        JOT_TRY(forward_body(m, m->canvas, B, L, st));
+        const int32_t* seq_map = nullptr;
+        if (compact && B_act < B) {
+            // finished sequences drop out of the forward pass: the batch is compacted to the live ones
+            launch_k(build_seq_map_kernel, dim3(1), dim3(32), 0, st, m->state, B, nb, m->seq_map, m->ctrl + 3);
+            JOT_TRY(launch_check());
+            seq_map = m->seq_map;
+        }
+        const int Bf = seq_map ? B_act : B;
+        JOT_TRY(forward_body(m, m->canvas, Bf, L, st, seq_map));
         {
             ProfScope ps(m, JOT_PROF_ROWS, st);
-            launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, m->canvas, B, L, m->cfg.mask_id, 0, 0, m->state, P, gen->block_len,
-                                                  nb, m->rows, m->ctrl + 1);
+            launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, m->canvas, Bf, L, m->cfg.mask_id, 0, 0, m->state, P,
+                     gen->block_len, nb, seq_map, m->rows, m->rows_out, m->ctrl + 1);
             JOT_TRY(launch_check());
-            launch_k(rmsnorm_kernel, dim3(B * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps,
-                                                  m->rows, m->ctrl + 1);
+            launch_k(rmsnorm_kernel, dim3(Bf * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model,
+                     m->cfg.rms_eps, m->rows, m->ctrl + 1);
             JOT_TRY(launch_check());
         }
         JOT_TRY(lm_head_from_hsel(m, gen->exclude_mask_token, d_bump_id, d_bump_val, m->g_top1, m->g_top2, m->g_sumexp,
-                                  m->g_argmax, B * gen->block_len, st));
+                                  m->g_argmax, Bf * gen->block_len, st));
         AcceptArgs a{};
         a.params = m->params_dev; a.per_seq_params = per_seq_params ? 1 : 0;
         a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
@@ -782,6 +798,7 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         JOT_CUDA(cudaStreamSynchronize(st));
         if (m->h_pinned[0]) return JOT_ERR_TIMEOUT;
         if (m->h_pinned[2] == 0) break;
+        B_act = m->h_pinned[2];
     }
     JOT_CUDA(cudaMemcpyAsync(d_out_tokens, m->canvas, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
     SeqState* hs = reinterpret_cast<SeqState*>(m->h_pinned + 16);

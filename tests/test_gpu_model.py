@@ -124,6 +124,9 @@ def test_generate_batch_equals_separate_runs(jot):
         assert torch.equal(o1[0], out[b]) and u1[0] == used[b]
     # the planted bump makes sequences stop early at different steps
     assert min(used) < T
+    # finished sequences dropping out of the forward pass changes nothing but the work done
+    out_nc, used_nc, passes_nc = model.generate(prompt, G, T, jp, 8, bump_id=ids, bump_val=val, compact_finished=False)
+    assert torch.equal(out, out_nc) and used == used_nc and passes == passes_nc
     # same call twice: identical result
     out2, used2, _ = model.generate(prompt, G, T, jp, 8, bump_id=ids, bump_val=val)
     assert torch.equal(out, out2) and used == used2
@@ -132,6 +135,26 @@ def test_generate_batch_equals_separate_runs(jot):
     out3, used3, _ = model.generate(prompt, G, T, pl, 8, bump_id=ids, bump_val=val)
     assert used3[0] == G // 8 and used3[1] == T and used3[2] == used[2]
     assert torch.equal(out3[2], out[2])
+    model.close()
+
+
+def test_finished_sequences_drop_out_of_the_batch(jot):
+    """Five sequences with very different thresholds finish at different steps; compacting the batch to the
+    live sequences must not change any token or step count (rows of a projection do not depend on which
+    other rows share the launch)."""
+    g = GEOMS["gqa"]
+    P, G, T, B = 24, 64, 64, 5
+    w_gpu = inputs.weights_to(inputs.model_weights(g, seed=0), "cuda")
+    prompt = inputs.prompt(8, B, P, g.vocab, g.mask_id).cuda()
+    ids, val = inputs.logit_bump(8, B, P + G, g.vocab, g.mask_id, hi=14.0, device="cuda")
+    model = jot.Model(g, w_gpu, B, P + G)
+    pl = [jot.Params(0.0, 0.0, 0.5, 8), jot.Params(30.0, 1.0, 0.5, 8), jot.Params(float("inf"), float("inf"), 0.5, 8),
+          jot.Params(5.0, 1.0, 0.9, 16), jot.Params(90.0, 1.0, 0.5, 8)]
+    on = model.generate(prompt, G, T, pl, 16, bump_id=ids, bump_val=val, compact_finished=True)
+    off = model.generate(prompt, G, T, pl, 16, bump_id=ids, bump_val=val, compact_finished=False)
+    assert torch.equal(on[0], off[0]) and on[1] == off[1] and on[2] == off[2]
+    used = on[1]
+    assert used[0] == G // 16 and used[2] == T and len(set(used)) >= 3 and (on[0] != g.mask_id).all()
     model.close()
 
 
