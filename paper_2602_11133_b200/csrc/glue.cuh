@@ -102,19 +102,37 @@ __global__ void rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_b
     }
 }
 
-// Split-K tail fused with the next RMSNorm: one CTA per row.
+// Split-K tail fused with the next RMSNorm: one CTA per row, one (at most two) 8-element vectors per thread,
+// every load of a thread issued before the first use so that a row costs one round trip to L2.
 //   h[row, :]   = bf16( sum over K ranges of partial + residual )          (the projection's output)
 //   out[row, :] = bf16( h * rsqrt(mean(h^2) + eps) * gain )                (h as rounded, like rmsnorm_kernel)
-// N multiple of 8, N/8 <= 8 * blockDim.x.
-__global__ void splitk_reduce_norm_kernel(const float* __restrict__ partial, int split, const __nv_bfloat16* residual,
-                                          __nv_bfloat16* C, int M, int N, const __nv_bfloat16* __restrict__ gain,
-                                          __nv_bfloat16* __restrict__ out, float eps) {
+// N multiple of 8, N/8 <= 2 * blockDim.x (at most 512 threads), split <= 4.
+__global__ void __launch_bounds__(512) splitk_reduce_norm_kernel(const float* __restrict__ partial, int split,
+                                                                  const __nv_bfloat16* residual, __nv_bfloat16* C, int M,
+                                                                  int N, const __nv_bfloat16* __restrict__ gain,
+                                                                  __nv_bfloat16* __restrict__ out, float eps) {
     grid_launch_dependents();
     grid_dependency_wait();
     __shared__ float scratch[33];
     const int row = blockIdx.x, nvec = N / 8;
     const size_t total = (size_t)M * N, base = (size_t)row * N;
-    constexpr int MAXV = 8;
+    constexpr int MAXV = 2, MAXS = 4;
+    float4 pa[MAXV][MAXS][2];
+    uint4 rv[MAXV], gv[MAXV];
+#pragma unroll
+    for (int t = 0; t < MAXV; ++t) {
+        const int i = threadIdx.x + t * blockDim.x;
+        if (i < nvec) {
+#pragma unroll
+            for (int s = 0; s < MAXS; ++s)
+                if (s < split) {
+                    pa[t][s][0] = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8);
+                    pa[t][s][1] = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8 + 4);
+                }
+            rv[t] = residual ? *reinterpret_cast<const uint4*>(residual + base + i * 8) : make_uint4(0, 0, 0, 0);
+            gv[t] = *reinterpret_cast<const uint4*>(gain + i * 8);
+        }
+    }
     uint4 hbuf[MAXV];
     float ss = 0.f;
 #pragma unroll
@@ -124,43 +142,34 @@ __global__ void splitk_reduce_norm_kernel(const float* __restrict__ partial, int
             float x[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) x[j] = 0.f;
-            for (int s = 0; s < split; ++s) {
-                const float4 a = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8);
-                const float4 b = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8 + 4);
-                x[0] += a.x; x[1] += a.y; x[2] += a.z; x[3] += a.w;
-                x[4] += b.x; x[5] += b.y; x[6] += b.z; x[7] += b.w;
-            }
-            if (residual) {
-                const uint4 rv = *reinterpret_cast<const uint4*>(residual + base + i * 8);
-                const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float2 f = __bfloat1622float2(r2[j]);
-                    x[2 * j] += f.x;
-                    x[2 * j + 1] += f.y;
+            for (int s = 0; s < MAXS; ++s)
+                if (s < split) {
+                    const float4 a = pa[t][s][0], b = pa[t][s][1];
+                    x[0] += a.x; x[1] += a.y; x[2] += a.z; x[3] += a.w;
+                    x[4] += b.x; x[5] += b.y; x[6] += b.z; x[7] += b.w;
                 }
-            }
+            const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rv[t]);
             __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&hbuf[t]);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                o2[j] = __floats2bfloat162_rn(x[2 * j], x[2 * j + 1]);
-                const float2 f = __bfloat1622float2(o2[j]);
-                ss += f.x * f.x + f.y * f.y;
+                const float2 f = __bfloat1622float2(r2[j]);        // zero when there is no residual
+                o2[j] = __floats2bfloat162_rn(x[2 * j] + f.x, x[2 * j + 1] + f.y);
+                const float2 hr = __bfloat1622float2(o2[j]);
+                ss += hr.x * hr.x + hr.y * hr.y;
             }
             *reinterpret_cast<uint4*>(C + base + i * 8) = hbuf[t];
         }
     }
     ss = block_sum(ss, scratch);
     const float inv = rsqrtf(ss / (float)N + eps);
-    const uint4* g4 = reinterpret_cast<const uint4*>(gain);
 #pragma unroll
     for (int t = 0; t < MAXV; ++t) {
         const int i = threadIdx.x + t * blockDim.x;
         if (i < nvec) {
-            const uint4 gv = g4[i];
             uint4 ov;
             const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&hbuf[t]);
-            const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gv);
+            const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gv[t]);
             __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {

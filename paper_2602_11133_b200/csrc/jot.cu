@@ -209,9 +209,11 @@ int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, 
             p.partial = scratch;
             const long items = (long)((p.M + 127) / 128) * ((p.N + 255) / 256) * split;
             JOT_TRY((launch_gemm_t<256, EPI_PARTIAL>(p, tmA, w.m256, (int)items, st)));
-            if (norm && p.ldc == p.N && p.N / 8 <= 8 * 256) {
-                launch_k(splitk_reduce_norm_kernel, dim3(p.M), dim3(256), 0, st, scratch, split, p.residual, p.C, p.M, p.N,
-                         norm->gain, norm->out, norm->eps);
+            if (norm && p.ldc == p.N && p.N / 8 <= 1024) {
+                int threads = (p.N / 8 + 31) / 32 * 32;      // one 8-element vector per thread up to 512 threads
+                threads = threads > 512 ? 512 : (threads < 64 ? 64 : threads);
+                launch_k(splitk_reduce_norm_kernel, dim3(p.M), dim3(threads), 0, st, scratch, split, p.residual, p.C, p.M,
+                         p.N, norm->gain, norm->out, norm->eps);
                 norm->done = true;
                 return launch_check();
             }
