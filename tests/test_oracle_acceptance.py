@@ -175,6 +175,18 @@ def test_accept_or_with_schedule_uncapped():
     assert x == [7, 7, 7, 7, 204, 205, 206, 207, 208, 209] and len(rep.exited) == 6
 
 
+def test_decision_is_inclusive():
+    # Eq. 8 is r >= tau: a ratio exactly on the threshold exits
+    st = jo.RowStats(m1=0.0, i1=5, m2=math.log(0.5), S=2.0)           # p1 = 0.5, p2 = 0.25, r = 2 exactly
+    assert jo.confidence_ratio(st.p1, st.p2, 0.0) == 2.0
+    x = canvas("mm")
+    rep = jo.accept_freeze(x, {0: st, 1: st}, jo.JotParams(2.0, 2.0, 0.5, 8, eps=0.0), M, 0, 2, 0)
+    assert rep.exited == [0, 1] and x == [5, 5]
+    x = canvas("mm")
+    rep = jo.accept_freeze(x, {0: st, 1: st}, jo.JotParams(2.0000002, 2.0000002, 0.5, 8, eps=0.0), M, 0, 2, 0)
+    assert rep.exited == [] and x == [M, M]
+
+
 def test_schedule_ties_and_alternative_reading():
     x = canvas("mmmm")
     stats = {i: stats_from_gap(50 + i, 0.1, p1=0.5) for i in range(4)}
