@@ -372,7 +372,7 @@ def run_model(args, jot, dev, world, rank, peaks, peaks_kind, config, g, nl, B, 
     line["generated_tokens_per_s"] = round(world * B * (host_out.shape[1] - P) / (e2e_ms_max / 1e3), 2)
     line["e2e"] = {"value": round(world * passes / (e2e_ms_max / 1e3), 3), "unit": "steps/s",
                    "h2d_bytes_per_step": round(prompt_host.numel() * 4 / max(passes, 1), 2),
-                   "d2h_bytes_per_step": round(host_out.numel() * 4 / max(passes, 1) + 12, 2),
+                   "d2h_bytes_per_step": round(host_out.numel() * 4 / max(passes, 1) + 16, 2),
                    "call": "jot_generate: pinned host prompt in, host tokens out (whole generation)",
                    "forward_passes": passes, "steps_used": used,
                    "generation": f"{e2e_G} tokens, up to {e2e_T} steps" + (" (shortened)" if (e2e_G, e2e_T) != (G, T) else "")}

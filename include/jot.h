@@ -206,6 +206,12 @@ enum {
 int jot_profile(jot_model* m, int enable);
 int jot_profile_read(jot_model* m, double* ms, int64_t* launches, int n_classes);
 
+/* Failure-path self test.  Every device-side wait in this library is bounded in wall time and, on expiry,
+ * makes the kernel unwind and set a status word instead of hanging.  This launches a one-CTA kernel that waits
+ * (for at most limit_ns nanoseconds, <= 5e9) on a barrier nothing ever signals and writes 1 to *d_status when
+ * the wait gives up, 0 if it did not.  The kernel ends normally and the context stays usable. */
+int jot_selftest_wait_expiry(int32_t* d_status, uint64_t limit_ns, void* stream);
+
 /* Number of kernels this library has launched from the calling process so far. */
 int64_t jot_launch_count(void);
 

@@ -41,7 +41,10 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bflo
     grid_dependency_wait();
     const int row = blockIdx.x;
     int src_row = row;
-    if (seq_map) src_row = seq_map[row / L] * L + row % L;
+    if (seq_map) {
+        const int b = seq_map[row / L];                 // unused slots (-1) compute on sequence 0; nobody reads them
+        src_row = (b < 0 ? 0 : b) * L + row % L;
+    }
     const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[src_row] * d);
     uint4* dst = reinterpret_cast<uint4*>(h + (size_t)row * d);
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = src[i];
@@ -201,6 +204,7 @@ __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restr
     __syncthreads();
     for (int slot = 0; slot < B; ++slot) {
         const int b = seq_map ? seq_map[slot] : slot;
+        if (b < 0) continue;                                // unused slot of a compacted batch
         int lo = blk_lo, hi = blk_hi;
         if (state) {
             const int blk = state[b].blk;
@@ -287,7 +291,8 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
     }
 }
 
-// Sequences that still have work, in ascending order: seq_map[slot] = b, *n_active = count.  One warp.
+// Sequences that still have work, in ascending order: seq_map[slot] = b, the remaining slots -1,
+// *n_active = count.  One warp.
 __global__ void build_seq_map_kernel(const SeqState* __restrict__ state, int B, int n_blocks,
                                      int32_t* __restrict__ seq_map, int32_t* __restrict__ n_active) {
     grid_launch_dependents();
@@ -301,6 +306,7 @@ __global__ void build_seq_map_kernel(const SeqState* __restrict__ state, int B, 
         if (live) seq_map[total + __popc(bal & ((1u << ln) - 1u))] = b;
         total += __popc(bal);
     }
+    for (int slot = total + ln; slot < B; slot += 32) seq_map[slot] = -1;
     if (ln == 0) *n_active = total;
 }
 

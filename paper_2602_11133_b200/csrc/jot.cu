@@ -293,7 +293,8 @@ struct jot_model {
     // activation tensor maps, re-encoded when (B, L) changes
     int map_B = -1, map_L = -1;
     CUtensorMap tm_a, tm_attn, tm_act, tm_hsel, tm_qkv3, tm_vt;
-    int32_t* h_pinned = nullptr;    // pinned host words for loop control read-back
+    int32_t* h_pinned = nullptr;    // pinned host words for loop control read-back (two 4-word slots, then SeqState)
+    cudaEvent_t step_done[2] = {nullptr, nullptr};
     // optional per-kernel-class timing with CUDA events on the launching stream
     bool profiling = false;
     std::vector<cudaEvent_t> ev_pool;
@@ -509,6 +510,23 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     return launch_check();
 }
 
+// One CTA waits on an mbarrier that nothing ever arms, through the same bounded wait every kernel uses, and
+// reports that the wait gave up.  The kernel returns normally: the context stays usable.
+__global__ void wait_expiry_kernel(int32_t* status, unsigned long long limit_ns) {
+    __shared__ uint64_t never_armed;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&never_armed, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = mbar_wait(&never_armed, 0, &abort_flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0) status[0] = ok ? 0 : (abort_flag ? 1 : 2);
+}
+
 // copy rows of a [*, d] bf16 matrix selected by `rows` (only r < *d_R)
 __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int d,
                                    const int32_t* __restrict__ rows, const int32_t* __restrict__ d_R) {
@@ -624,6 +642,7 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
 
     int rc = JOT_OK;
     auto fail = [&](int code) {
+        for (cudaEvent_t ev : m->step_done) if (ev) cudaEventDestroy(ev);
         if (m->h_pinned) cudaFreeHost(m->h_pinned);
         delete m;
         return code;
@@ -658,6 +677,7 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
     if (e == cudaSuccess) e = cudaMemset(m->hsel, 0, (size_t)m->R_cap * d * 2);
     if (e == cudaSuccess) e = cudaMemset(m->rows, 0, (size_t)m->R_cap * 4);
     if (e == cudaSuccess) e = cudaMemset(m->rows_out, 0, (size_t)m->R_cap * 4);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&m->step_done[i], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaHostAlloc((void**)&m->h_pinned, 64 + (size_t)max_batch * sizeof(SeqState), cudaHostAllocDefault);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
@@ -670,6 +690,7 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
 int jot_free_model(jot_model* m) {
     if (!m) return JOT_ERR_ARG;
     if (m->h_pinned) cudaFreeHost(m->h_pinned);
+    for (cudaEvent_t ev : m->step_done) if (ev) cudaEventDestroy(ev);
     for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
     delete m;
     return JOT_OK;
@@ -759,10 +780,22 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     launch_k(init_canvas_kernel, dim3((B * L + 255) / 256), dim3(256), 0, st, d_prompt, m->canvas, B, P, gen->gen_len, m->cfg.mask_id,
                                                            m->state);
     JOT_TRY(launch_check());
+    // The host runs one step ahead of what it knows: step `it` is enqueued before the outcome of step it-1 has
+    // been read, so the GPU never idles while the host looks at the loop condition.  A step enqueued after the
+    // last sequence finished finds nothing masked and changes nothing; it is not counted.
     int passes = 0;
-    int B_act = B;                                   // sequences that still have work (known from the last step)
+    int B_act = B;                                   // upper bound on the sequences that still have work
     const bool compact = gen->compact_finished != 0;
-    for (int it = 0; it < gen->steps; ++it) {
+    auto outcome = [&](int slot, bool* finished) -> int {      // wait for a step's control words
+        JOT_CUDA(cudaEventSynchronize(m->step_done[slot]));
+        const int32_t* w = m->h_pinned + 4 * slot;
+        if (w[0]) return JOT_ERR_TIMEOUT;
+        *finished = w[2] == 0;
+        if (!*finished) B_act = w[2];
+        return JOT_OK;
+    };
+    bool finished = false;
+    for (int it = 0; it < gen->steps && !finished; ++it) {
         JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
         const int32_t* seq_map = nullptr;
         if (compact && B_act < B) {
@@ -795,12 +828,14 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
             ProfScope ps(m, JOT_PROF_ACCEPT, st);
             JOT_TRY(launch_accept(a, st));
         }
+        JOT_CUDA(cudaMemcpyAsync(m->h_pinned + 4 * (it & 1), m->ctrl, 16, cudaMemcpyDeviceToHost, st));
+        JOT_CUDA(cudaEventRecord(m->step_done[it & 1], st));
+        if (it >= 1) {
+            JOT_TRY(outcome((it - 1) & 1, &finished));       // step it-1; step `it` is already in flight
+            if (finished) break;                              // ... and was a no-op
+        }
         ++passes;
-        JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 12, cudaMemcpyDeviceToHost, st));
-        JOT_CUDA(cudaStreamSynchronize(st));
-        if (m->h_pinned[0]) return JOT_ERR_TIMEOUT;
-        if (m->h_pinned[2] == 0) break;
-        B_act = m->h_pinned[2];
+        if (it == gen->steps - 1) JOT_TRY(outcome(it & 1, &finished));
     }
     JOT_CUDA(cudaMemcpyAsync(d_out_tokens, m->canvas, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
     SeqState* hs = reinterpret_cast<SeqState*>(m->h_pinned + 16);
@@ -809,6 +844,12 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     for (int b = 0; b < B; ++b) h_steps_used[b] = hs[b].steps_used;
     if (h_forward_passes) *h_forward_passes = passes;
     return JOT_OK;
+}
+
+int jot_selftest_wait_expiry(int32_t* d_status, uint64_t limit_ns, void* stream) {
+    if (!d_status || limit_ns == 0 || limit_ns > 5000000000ull) return JOT_ERR_ARG;
+    wait_expiry_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(d_status, (unsigned long long)limit_ns);
+    return launch_check();
 }
 
 int jot_profile(jot_model* m, int enable) {

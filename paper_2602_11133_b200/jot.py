@@ -20,6 +20,7 @@ EXPORTS = [
     "jot_status_string", "jot_last_cuda_error", "jot_workspace_bytes", "jot_init_model", "jot_free_model",
     "jot_denoise_step", "jot_lm_head_stats", "jot_accept_freeze", "jot_generate", "jot_gemm_bf16",
     "jot_launch_count", "jot_profile", "jot_profile_read", "jot_gemm_bf16_noalloc",
+    "jot_selftest_wait_expiry",
 ]
 
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -96,6 +97,7 @@ def _lib():
         lib.jot_gemm_bf16_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                               C.c_void_p, C.c_void_p]
         lib.jot_launch_count.restype = C.c_int64
+        lib.jot_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         lib.jot_profile.argtypes = [C.c_void_p, C.c_int]
         lib.jot_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int]
         _LIB = lib
@@ -286,3 +288,10 @@ def gemm_bf16_noalloc(a: torch.Tensor, w: torch.Tensor, residual: Optional[torch
                                         M, N, K, _ptr(status, torch.int32, "status"), _stream()),
            "jot_gemm_bf16_noalloc")
     return out
+
+
+def selftest_wait_expiry(limit_ns: int = 20_000_000) -> int:
+    """Run the bounded-wait self test; returns the status word the kernel wrote (1 = the wait gave up)."""
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    _check(_lib().jot_selftest_wait_expiry(status.data_ptr(), limit_ns, _stream()), "jot_selftest_wait_expiry")
+    return int(status.item())

@@ -72,6 +72,18 @@ def test_gemm_residual_in_place(jot):
     assert (err <= 2.0 ** -8 * want.abs() + 1e-3 * want.abs().max()).all()
 
 
+def test_bounded_wait_gives_up_and_leaves_the_context_usable(jot):
+    """A wait on a barrier that nothing signals ends after its time limit with a status, not a hang."""
+    import time
+    t0 = time.perf_counter()
+    assert jot.selftest_wait_expiry(20_000_000) == 1
+    assert time.perf_counter() - t0 < 2.0
+    a = inputs.normal(1, "a", (128, 64), 1.0).cuda()
+    w = inputs.normal(1, "w", (256, 64), 0.05).cuda()
+    out = jot.gemm_bf16(a, w)                      # the context is still healthy
+    assert torch.isfinite(out.float()).all()
+
+
 # ---------------------------------------------------------------- acceptance / freeze
 def random_accept_case(seed, B, L, P, mask_id, V, hot=0.3):
     rng = np.random.default_rng(seed)
