@@ -87,11 +87,14 @@ typedef struct {
  * gen_len, and gen_len/block_len must divide steps).  exclude_mask_token != 0 keeps the mask token
  * out of the candidate predictions.  compact_finished: the paper decodes one sequence at a time, where
  * early stopping ends the loop; in a batch the loop runs until the slowest sequence is done, and with this
- * flag the forward pass only covers the sequences still decoding (same tokens and step counts, fewer rows). */
+ * flag the forward pass only covers the sequences still decoding (same tokens and step counts, fewer rows).
+ * use_cuda_graph: the kernels of one step are captured on `stream` (which therefore must not already be
+ * capturing) and replayed as one graph launch per step; pays off when a step is a few dozen short kernels. */
 typedef struct {
     int32_t gen_len, steps, block_len;
     int32_t exclude_mask_token;
     int32_t compact_finished;   /* != 0: sequences that have finished drop out of later forward passes */
+    int32_t use_cuda_graph;     /* != 0: a step is captured into a CUDA graph once and replayed */
 } jot_gen_config;
 
 typedef struct jot_model jot_model; /* opaque; host-side object owned by the library */

@@ -794,17 +794,14 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         if (!*finished) B_act = w[2];
         return JOT_OK;
     };
-    bool finished = false;
-    for (int it = 0; it < gen->steps && !finished; ++it) {
+    // everything one step enqueues, ending with the copy of the control words to the pinned slot it & 1
+    auto enqueue_step = [&](int it, int Bf, const int32_t* seq_map) -> int {
         JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
-        const int32_t* seq_map = nullptr;
-        if (compact && B_act < B) {
+        if (seq_map) {
             // finished sequences drop out of the forward pass: the batch is compacted to the live ones
             launch_k(build_seq_map_kernel, dim3(1), dim3(32), 0, st, m->state, B, nb, m->seq_map, m->ctrl + 3);
             JOT_TRY(launch_check());
-            seq_map = m->seq_map;
         }
-        const int Bf = seq_map ? B_act : B;
         JOT_TRY(forward_body(m, m->canvas, Bf, L, st, seq_map));
         {
             ProfScope ps(m, JOT_PROF_ROWS, st);
@@ -821,7 +818,7 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         a.params = m->params_dev; a.per_seq_params = per_seq_params ? 1 : 0;
         a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
         a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp; a.argmax = m->g_argmax;
-        a.step_index = it + 1;
+        a.step_index = it + 1;                       // only reaches the optional exit-step output, unused here
         a.state = m->state; a.P = P; a.block_len = gen->block_len; a.n_blocks = nb; a.steps_per_block = Tb;
         a.n_unfinished = m->ctrl + 2;
         {
@@ -829,18 +826,72 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
             JOT_TRY(launch_accept(a, st));
         }
         JOT_CUDA(cudaMemcpyAsync(m->h_pinned + 4 * (it & 1), m->ctrl, 16, cudaMemcpyDeviceToHost, st));
-        JOT_CUDA(cudaEventRecord(m->step_done[it & 1], st));
+        return JOT_OK;
+    };
+    // With use_cuda_graph the step is captured once per (batch size after compaction, pinned slot) and replayed:
+    // the step's few dozen launches become one graph launch, which is what a small model's step time consists of.
+    struct StepGraph { int Bf, slot; cudaGraphExec_t exec; int64_t launches; };
+    std::vector<StepGraph> graphs;
+    auto release_graphs = [&]() {
+        for (auto& g : graphs) cudaGraphExecDestroy(g.exec);
+        graphs.clear();
+    };
+    const bool want_graph = gen->use_cuda_graph != 0 && !m->profiling;
+    bool graph_ok = want_graph;
+    bool finished = false;
+    int rc = JOT_OK;
+    for (int it = 0; it < gen->steps && !finished; ++it) {
+        const int32_t* seq_map = (compact && B_act < B) ? m->seq_map : nullptr;
+        const int Bf = seq_map ? B_act : B;
+        bool launched = false;
+        if (graph_ok && it >= 1) {                   // step 0 runs eagerly (one-time attribute and map set-up)
+            StepGraph* g = nullptr;
+            for (auto& c : graphs) if (c.Bf == Bf && c.slot == (it & 1)) g = &c;
+            if (!g) {
+                cudaGraph_t graph = nullptr;
+                const int64_t before = g_launches.load();
+                if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+                    const int erc = enqueue_step(it, Bf, seq_map);
+                    const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+                    cudaGraphExec_t exec = nullptr;
+                    if (erc == JOT_OK && ce == cudaSuccess && graph &&
+                        cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+                        graphs.push_back({Bf, it & 1, exec, g_launches.load() - before});
+                        g = &graphs.back();
+                    }
+                    if (graph) cudaGraphDestroy(graph);
+                }
+                g_launches.store(before);            // captured launches are counted when the graph runs
+                if (!g) {                            // capture is unavailable: go on with plain launches
+                    cudaGetLastError();
+                    graph_ok = false;
+                }
+            }
+            if (g) {
+                if (cudaGraphLaunch(g->exec, st) != cudaSuccess) { rc = JOT_ERR_CUDA; g_last_cuda_error = (int)cudaGetLastError(); break; }
+                g_launches.fetch_add(g->launches);
+                launched = true;
+            }
+        }
+        if (!launched && (rc = enqueue_step(it, Bf, seq_map)) != JOT_OK) break;
+        if (cudaEventRecord(m->step_done[it & 1], st) != cudaSuccess) { rc = JOT_ERR_CUDA; break; }
         if (it >= 1) {
-            JOT_TRY(outcome((it - 1) & 1, &finished));       // step it-1; step `it` is already in flight
-            if (finished) break;                              // ... and was a no-op
+            if ((rc = outcome((it - 1) & 1, &finished)) != JOT_OK) break;   // step it-1; step `it` is already in flight
+            if (finished) break;                                             // ... and was a no-op
         }
         ++passes;
-        if (it == gen->steps - 1) JOT_TRY(outcome(it & 1, &finished));
+        if (it == gen->steps - 1 && (rc = outcome(it & 1, &finished)) != JOT_OK) break;
+    }
+    if (rc != JOT_OK) {
+        cudaStreamSynchronize(st);
+        release_graphs();
+        return rc;
     }
     JOT_CUDA(cudaMemcpyAsync(d_out_tokens, m->canvas, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
     SeqState* hs = reinterpret_cast<SeqState*>(m->h_pinned + 16);
     JOT_CUDA(cudaMemcpyAsync(hs, m->state, (size_t)B * sizeof(SeqState), cudaMemcpyDeviceToHost, st));
     JOT_CUDA(cudaStreamSynchronize(st));
+    release_graphs();
     for (int b = 0; b < B; ++b) h_steps_used[b] = hs[b].steps_used;
     if (h_forward_passes) *h_forward_passes = passes;
     return JOT_OK;

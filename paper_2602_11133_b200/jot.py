@@ -61,7 +61,7 @@ class _Weights(C.Structure):
 
 class GenConfig(C.Structure):
     _fields_ = [("gen_len", C.c_int32), ("steps", C.c_int32), ("block_len", C.c_int32),
-                ("exclude_mask_token", C.c_int32), ("compact_finished", C.c_int32)]
+                ("exclude_mask_token", C.c_int32), ("compact_finished", C.c_int32), ("use_cuda_graph", C.c_int32)]
 
 
 _LIB = None
@@ -222,7 +222,7 @@ class Model:
     # ---- Algorithm 1 ----------------------------------------------------------------------------
     def generate(self, prompt: torch.Tensor, gen_len: int, steps: int, params, block_len: Optional[int] = None,
                  exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
-                 bump_val: Optional[torch.Tensor] = None, compact_finished: bool = True):
+                 bump_val: Optional[torch.Tensor] = None, compact_finished: bool = True, use_cuda_graph: bool = False):
         """Returns (tokens [B, P+gen_len] int32 on device, steps_used list[int], forward_passes int)."""
         B, P = prompt.shape
         per_seq = isinstance(params, (list, tuple))
@@ -232,7 +232,8 @@ class Model:
             parr = (Params * B)(*params)
         else:
             parr = (Params * 1)(params)
-        gen = GenConfig(gen_len, steps, block_len or gen_len, int(exclude_mask_token), int(compact_finished))
+        gen = GenConfig(gen_len, steps, block_len or gen_len, int(exclude_mask_token), int(compact_finished),
+                        int(use_cuda_graph))
         out = torch.empty(B, P + gen_len, dtype=torch.int32, device=prompt.device)
         used = (C.c_int32 * B)()
         passes = C.c_int32(0)

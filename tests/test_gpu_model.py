@@ -127,6 +127,9 @@ def test_generate_batch_equals_separate_runs(jot):
     # finished sequences dropping out of the forward pass changes nothing but the work done
     out_nc, used_nc, passes_nc = model.generate(prompt, G, T, jp, 8, bump_id=ids, bump_val=val, compact_finished=False)
     assert torch.equal(out, out_nc) and used == used_nc and passes == passes_nc
+    # replaying the step as a CUDA graph changes nothing either
+    out_g, used_g, passes_g = model.generate(prompt, G, T, jp, 8, bump_id=ids, bump_val=val, use_cuda_graph=True)
+    assert torch.equal(out, out_g) and used == used_g and passes == passes_g
     # same call twice: identical result
     out2, used2, _ = model.generate(prompt, G, T, jp, 8, bump_id=ids, bump_val=val)
     assert torch.equal(out, out2) and used == used2
