@@ -40,12 +40,18 @@ import numpy as np
 
 @dataclasses.dataclass(frozen=True)
 class JotParams:
-    """tau_max, tau_min, gamma, D of Algorithm 1; eps of Eq. 4 (1e-12, Section 4.2)."""
+    """tau_max, tau_min, gamma, D of Algorithm 1; eps of Eq. 4 (1e-12, Section 4.2).
+
+    gate = "ratio" is the paper's test r >= tau (Eq. 8).  gate = "maxprob" is the fixed probability gate the
+    paper contrasts it with (Section 2: a position is finalised when its max probability clears a threshold,
+    0.9 in the compared system): p1 >= prob_threshold, no spatial modulation."""
     tau_max: float = 90.0
     tau_min: float = 1.0
     gamma: float = 0.5
     D: int = 8
     eps: float = 1e-12
+    gate: str = "ratio"
+    prob_threshold: float = 0.9
 
 
 DREAM_DEFAULT = JotParams(90.0, 1.0, 0.5, 8)   # Table 1 caption
@@ -88,6 +94,72 @@ def row_stats(logits: np.ndarray, mask_id: Optional[int] = None) -> RowStats:
 def confidence_ratio(p1: float, p2: float, eps: float = 1e-12) -> float:
     """Eq. 4: r = p1 / (p2 + eps)."""
     return p1 / (p2 + eps)
+
+
+# ----------------------------------------------------------------------------
+# Section 4.1, "Early-Exit Decision": the finalised token may be sampled from pi instead of argmax
+# ----------------------------------------------------------------------------
+_M64 = (1 << 64) - 1
+_GOLDEN = 0x9E3779B97F4A7C15
+
+
+def _mix64(z: int) -> int:
+    """Output function of splitmix64 (Steele, Lea, Flood 2014; Vigna's reference implementation)."""
+    z &= _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def splitmix64_output(state0: int, n: int) -> int:
+    """n-th output (n >= 1) of the splitmix64 stream whose state starts at state0."""
+    return _mix64(state0 + n * _GOLDEN)
+
+
+def gumbel_key(seed: int, step: int, flat_pos: int) -> int:
+    """Start state of the stream that serves one (step, canvas position): a mix of the three numbers."""
+    return _mix64((seed ^ (step << 40) ^ flat_pos) & _M64)
+
+
+def sample_token(logits: np.ndarray, mask_id: Optional[int], temperature: float, seed: int, step: int,
+                 flat_pos: int) -> int:
+    """Draw from softmax(l / temperature) by the Gumbel-max identity: argmax_v (l_v / T + G_v), G_v = -ln(-ln u_v).
+
+    u_v comes from a counter-based generator so that any implementation can reproduce the draw: the top 23
+    bits k of output number v + 1 of the splitmix64 stream keyed by (seed, step, position) give
+    u = (k + 0.5) / 2^23.  Ties resolve to the lowest token id; the mask column is not a candidate."""
+    l = np.asarray(logits, dtype=np.float64)
+    key = gumbel_key(seed, step, flat_pos)
+    best, best_v = -math.inf, -1
+    inv_t = 1.0 / temperature
+    for v in range(l.shape[0]):
+        if v == mask_id:
+            continue
+        k = splitmix64_output(key, v + 1) >> 41
+        u = (k + 0.5) / float(1 << 23)
+        score = l[v] * inv_t - math.log(-math.log(u))
+        if score > best:
+            best, best_v = score, v
+    return best_v
+
+
+def sample_tokens_fast(logits: np.ndarray, mask_id: Optional[int], temperature: float, seed: int, step: int,
+                       flat_pos: int) -> Tuple[int, float]:
+    """Same draw as sample_token with numpy integer arithmetic (for vocabularies of 1e5 entries); also returns
+    the gap between the two largest perturbed scores (a draw decided by less than rounding noise is a tie)."""
+    l = np.asarray(logits, dtype=np.float64)
+    key = np.uint64(gumbel_key(seed, step, flat_pos))
+    with np.errstate(over="ignore"):
+        z = key + (np.arange(1, l.shape[0] + 1, dtype=np.uint64)) * np.uint64(_GOLDEN)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        z = z ^ (z >> np.uint64(31))
+    u = ((z >> np.uint64(41)).astype(np.float64) + 0.5) / float(1 << 23)
+    score = l / temperature - np.log(-np.log(u))
+    if mask_id is not None:
+        score[mask_id] = -np.inf
+    order = np.argsort(-score, kind="stable")
+    return int(order[0]), float(score[order[0]] - score[order[1]])
 
 
 # ----------------------------------------------------------------------------
@@ -148,10 +220,11 @@ class StepReport:
 
 
 def accept_freeze(x: List[int], stats: dict, p: JotParams, mask_id: int, blk_lo: int, blk_hi: int,
-                  k_transfer: int, schedule_after_exit: bool = False) -> StepReport:
+                  k_transfer: int, schedule_after_exit: bool = False, tokens: Optional[dict] = None) -> StepReport:
     """Update one sequence in place.  `stats[i]` is a RowStats for every masked i in [blk_lo, blk_hi).
 
-    All decisions use the canvas and the statistics as they were at the start of the step.
+    All decisions use the canvas and the statistics as they were at the start of the step.  `tokens[i]`, when
+    given, is the token a finalised position receives (a sample from pi) instead of its argmax.
     """
     x0 = list(x)
     A = [i for i in range(blk_lo, blk_hi) if x0[i] == mask_id]          # Algorithm 1: M_n (in block)
@@ -162,6 +235,12 @@ def accept_freeze(x: List[int], stats: dict, p: JotParams, mask_id: int, blk_lo:
         r = confidence_ratio(st.p1, st.p2, p.eps)                         # Eq. 4
         t = position_threshold(x0, i, mask_id, p)                         # Eq. 5-7
         ratio[i], tau[i] = r, t
+        if p.gate == "maxprob":                                           # fixed probability gate (Section 2)
+            if abs(st.p1 - p.prob_threshold) <= 1e-3 * p.prob_threshold:
+                near.append(i)
+            if np.float32(st.p1) >= np.float32(p.prob_threshold):
+                E.append(i)
+            continue
         if abs(r - t) <= 1e-3 * abs(t):
             near.append(i)
         if np.float32(r) >= np.float32(t):                                # Eq. 8, decided in float32
@@ -171,7 +250,7 @@ def accept_freeze(x: List[int], stats: dict, p: JotParams, mask_id: int, blk_lo:
     ranked = sorted(cand, key=lambda i: (-stats[i].p1, i))                # highest max-prob, ties -> lower i
     U = sorted(ranked[:k])
     for i in set(E) | set(U):                                             # logical OR, uncapped
-        x[i] = stats[i].i1                                                # finalise by argmax
+        x[i] = stats[i].i1 if tokens is None else tokens[i]               # finalise by argmax (or by the sample)
     return StepReport(E, U, near, ratio, tau)
 
 
@@ -191,11 +270,15 @@ class Trajectory:
 def generate(logits_fn: Callable[[List[int], List[int]], dict], prompt: Sequence[int], gen_len: int,
              steps: int, p: JotParams, mask_id: int, block_len: Optional[int] = None,
              exclude_mask_token: bool = True, schedule_after_exit: bool = False,
-             stats_fn: Optional[Callable[[List[int], List[int]], dict]] = None) -> Trajectory:
+             stats_fn: Optional[Callable[[List[int], List[int]], dict]] = None,
+             sampling: Optional[Tuple[float, int]] = None, seq_index: int = 0) -> Trajectory:
     """Algorithm 1 for one sequence.
 
     logits_fn(x, rows) returns {i: logits row (length K)} for the requested masked positions;
     alternatively stats_fn(x, rows) returns {i: RowStats} directly (for stub models in tests).
+    sampling = (temperature, seed): finalised positions receive a sample from softmax(l / temperature) drawn
+    with sample_tokens_fast, keyed by the 0-based index of the forward pass and the position's flat canvas
+    index seq_index * L + i; the acceptance decisions themselves do not change.
     """
     P = len(prompt)
     Lb = gen_len if block_len is None else block_len
@@ -212,14 +295,18 @@ def generate(logits_fn: Callable[[List[int], List[int]], dict], prompt: Sequence
             A = [i for i in range(lo, hi) if x[i] == mask_id]             # M_n
             if not A:                                                     # break when nothing is masked
                 break
+            drawn = None
             if stats_fn is not None:
                 stats = stats_fn(x, A)
             else:
                 rows = logits_fn(x, A)
                 stats = {i: row_stats(rows[i], mask_id if exclude_mask_token else None) for i in A}
+                if sampling is not None:
+                    drawn = {i: sample_tokens_fast(rows[i], mask_id if exclude_mask_token else None, sampling[0],
+                                                   sampling[1], traj.steps_used, seq_index * len(x) + i)[0] for i in A}
             traj.canvases.append(list(x))
             traj.blocks.append((lo, hi))
-            rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[s], schedule_after_exit)
+            rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[s], schedule_after_exit, drawn)
             traj.reports.append(rep)
             traj.steps_used += 1
             for i in set(rep.exited) | set(rep.scheduled):

@@ -294,3 +294,48 @@ def test_generate_with_logits_fn_excludes_mask_token():
 def test_reversal_budget_number():
     # Section 5 (theory): 2 * 256 / (1 + 90) is "about 5.6"
     assert 2 * 256 / 91 == pytest.approx(5.6, abs=0.05)
+
+
+# ---------------------------------------------------------------- sampling-based finalisation, probability gate
+def test_counter_generator_matches_published_splitmix64_vectors():
+    # first outputs of the reference implementation for seed 1234567
+    want = [6457827717110365317, 3203168211198807973, 9817491932198370423, 4593380528125082431, 16408922859458223821]
+    assert [jo.splitmix64_output(1234567, n) for n in range(1, 6)] == want
+
+
+def test_gumbel_max_draws_follow_the_softmax():
+    # chi-square of 20000 draws against softmax(l / T) on a 6-token vocabulary (mask column excluded)
+    l = np.array([1.0, 0.2, -0.5, 2.0, 50.0, 0.0])
+    mask = 4
+    for T in (1.0, 0.5):
+        p = np.exp(np.delete(l, mask) / T)
+        p /= p.sum()
+        counts = np.zeros(6)
+        n = 20000
+        for step in range(n):
+            counts[jo.sample_token(l, mask, T, seed=7, step=step, flat_pos=3)] += 1
+        assert counts[mask] == 0
+        c = np.delete(counts, mask)
+        chi2 = float(((c - n * p) ** 2 / (n * p)).sum())
+        assert chi2 < 20.5, (T, chi2)             # 4 degrees of freedom: P(chi2 > 20.5) < 4e-4
+    # the fast version is the same draw
+    for step in range(200):
+        assert jo.sample_tokens_fast(l, mask, 0.7, 11, step, 5)[0] == jo.sample_token(l, mask, 0.7, 11, step, 5)
+    # temperature -> 0 recovers the argmax; different positions and steps get different streams
+    assert all(jo.sample_token(l, mask, 1e-3, 1, s, 0) == 3 for s in range(50))
+    assert len({jo.gumbel_key(1, s, q) for s in range(20) for q in range(20)}) == 400
+
+
+def test_sampled_token_is_what_a_finalised_position_receives():
+    x = canvas("rrmm")
+    stats = {2: stats_from_gap(50, 10.0), 3: stats_from_gap(51, 0.01, p1=0.1)}
+    rep = jo.accept_freeze(x, stats, jo.DREAM_DEFAULT, M, 2, 4, 0, tokens={2: 77, 3: 78})
+    assert rep.exited == [2] and x == [7, 7, 77, M]            # decisions unchanged, token replaced
+
+
+def test_probability_gate():
+    x = canvas("rrmmm")
+    stats = {2: stats_from_gap(60, 0.1, p1=0.95), 3: stats_from_gap(61, 9.0, p1=0.5), 4: stats_from_gap(62, 0.1, p1=0.9)}
+    p = jo.JotParams(gate="maxprob", prob_threshold=0.9)
+    rep = jo.accept_freeze(x, stats, p, M, 2, 5, 0)
+    assert rep.exited == [2, 4] and x == [7, 7, 60, M, 62]      # inclusive; a large ratio alone does not pass
