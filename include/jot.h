@@ -47,13 +47,20 @@ int jot_last_cuda_error(void);
  * Paper defaults (Table 1 caption; Section 4.2): (90, 1, 0.5, 8) for Dream, (30, 1, 0.5, 8) for
  * LLaDA, eps = 1e-12.  1 <= D <= 32, 0 < gamma < 1 is what Eq. 5 assumes; gamma is not checked.
  * schedule_after_exit = 0: the transfer schedule ranks all masked candidates and is OR-ed with the
- * early-exit mask (Section 4.2 "Implementation details"); 1: it ranks only what early exit left. */
+ * early-exit mask (Section 4.2 "Implementation details"); 1: it ranks only what early exit left.
+ * gate: JOT_GATE_RATIO is the paper's test r >= tau (Eq. 8).  JOT_GATE_MAXPROB replaces it by the fixed
+ * probability gate the paper contrasts JoT with (Section 2): p1 >= prob_threshold, no spatial modulation;
+ * the transfer schedule and the OR are unchanged.  0 < prob_threshold <= 1 is required then, any other
+ * gate value is refused (JOT_ERR_ARG). */
 typedef struct {
     float tau_max, tau_min, gamma;
     int32_t D;
     float eps;
     int32_t schedule_after_exit;
+    int32_t gate;            /* 0 = JOT_GATE_RATIO, 1 = JOT_GATE_MAXPROB */
+    float prob_threshold;    /* JOT_GATE_MAXPROB: finalise when p1 >= prob_threshold */
 } jot_params;
+enum { JOT_GATE_RATIO = 0, JOT_GATE_MAXPROB = 1 };
 
 /* Geometry of the denoiser f_theta (Algorithm 1 treats it as given).  Llama-style: RMSNorm,
  * rotate-half RoPE on absolute canvas positions, grouped-query attention without any mask, SwiGLU
@@ -95,7 +102,23 @@ typedef struct {
     int32_t exclude_mask_token;
     int32_t compact_finished;   /* != 0: sequences that have finished drop out of later forward passes */
     int32_t use_cuda_graph;     /* != 0: a step is captured into a CUDA graph once and replayed */
+    float temperature;          /* > 0: finalised positions receive a sample from softmax(l / temperature) */
+    uint32_t seed_lo, seed_hi;  /* the 64-bit seed of jot_sampling; the step is the forward pass index */
 } jot_gen_config;
+
+/* Sampling-based finalisation (Section 4.1, "Early-Exit Decision": the finalised token may be drawn from
+ * the predicted distribution instead of taken as its argmax).  temperature > 0 turns it on: next to the
+ * statistics, every active row also yields one draw from softmax(logits / temperature), made by the
+ * Gumbel-max identity argmax_v(l_v / T - ln(-ln u_v)) inside the LM-head epilogue.  u_v = (k + 0.5) / 2^23
+ * with k the top 23 bits of output number v + 1 of the splitmix64 stream whose start state is
+ * mix64(seed ^ (step << 40) ^ flat_position), flat_position = b * L + i, so a draw depends only on
+ * (seed, step, position, token) and can be reproduced anywhere.  The acceptance decisions still use the
+ * un-tempered logits; pass the sampled array instead of the argmax array to jot_accept_freeze. */
+typedef struct {
+    float temperature;   /* <= 0: off */
+    uint64_t seed;
+    int32_t step;        /* index of this forward pass (0-based) */
+} jot_sampling;
 
 typedef struct jot_model jot_model; /* opaque; host-side object owned by the library */
 
@@ -124,6 +147,7 @@ int jot_free_model(jot_model* m);
 int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi,
                      int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val,
                      float* d_top1_logit, float* d_top2_logit, float* d_sumexp, int32_t* d_argmax,
+                     const jot_sampling* sampling /* nullable */, int32_t* d_sampled /* [B, L], with sampling */,
                      void* stream);
 
 /* The LM head + statistics part of jot_denoise_step alone, on caller-supplied final hidden states
@@ -132,7 +156,8 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
 int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_tokens, int B, int L,
                       int blk_lo, int blk_hi, int exclude_mask_token, const int32_t* d_bump_id,
                       const float* d_bump_val, float* d_top1_logit, float* d_top2_logit,
-                      float* d_sumexp, int32_t* d_argmax, void* stream);
+                      float* d_sumexp, int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled,
+                      void* stream);
 
 /* Section 4.1 Eq. 4-8 and the state update of Algorithm 1 for one step, in place on d_tokens [B, L].
  * Candidates are the positions of [blk_lo, blk_hi) that hold mask_id.  For each: confidence ratio

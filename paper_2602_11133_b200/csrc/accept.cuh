@@ -19,6 +19,8 @@ struct AcceptParamsDev {     // mirrors jot_params
     int32_t D;
     float eps;
     int32_t schedule_after_exit;
+    int32_t gate;                // 0: ratio r >= tau (Eq. 8); 1: fixed probability gate p1 >= prob_threshold
+    float prob_threshold;
 };
 
 // Per-sequence loop state used by the generate loop (device resident).
@@ -49,6 +51,7 @@ struct AcceptArgs {
     SeqState* state;                 // [B] nullable
     int P, block_len, n_blocks, steps_per_block;
     int32_t* n_unfinished;           // device counter: += 1 per sequence that still has work (nullable)
+    int32_t* step_counter;           // device counter of forward passes, advanced once per launch (nullable)
 };
 
 // Dynamic shared memory: resolved bitmap words, candidate list, candidate sum-exp, candidate flags.
@@ -57,6 +60,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     grid_launch_dependents();
     grid_dependency_wait();
     const int L = a.L, b = blockIdx.x, tid = threadIdx.x;
+    if (a.step_counter && b == 0 && tid == 0) atomicAdd(a.step_counter, 1);
     const int n_words = (L + 31) / 32;
     uint32_t* res_bits = sh;                                   // [n_words + 2] resolved bitmap (padded)
     int* cand = reinterpret_cast<int*>(sh + n_words + 2);     // [L] candidate positions, ascending
@@ -142,7 +146,9 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
         const float phi = fminf(1.f, w * inv_wmax);                        // Eq. 6
         const float tau = prm.tau_max - (prm.tau_max - prm.tau_min) * phi; // Eq. 7
         cand_S[c] = S;
-        cand_flag[c] = (r >= tau) ? 1 : 0;                                  // Eq. 8
+        // Eq. 8; or the fixed probability gate the paper contrasts it with (p1 = 1/S, no spatial modulation)
+        const bool exit_now = prm.gate == 1 ? (1.f / S >= prm.prob_threshold) : (r >= tau);
+        cand_flag[c] = exit_now ? 1 : 0;
     }
     __syncthreads();
 

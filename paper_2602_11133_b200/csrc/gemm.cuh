@@ -53,6 +53,12 @@ struct GemmParams {
     const float* bump_val;
     int mask_col;                 // column to exclude, or -1
     float4* partials;             // [chunks][R_pad] (m1, bitcast i1, m2, S)
+    // sampling-based finalisation (inv_temperature > 0): each row also draws a token from softmax(l / T)
+    float inv_temperature;
+    unsigned long long sample_seed;
+    const int32_t* d_step;        // device step counter (nullable: then step_value)
+    int step_value;
+    float2* partials2;            // [chunks][R_pad] (best perturbed score, bitcast token)
     int R_pad;                    // row capacity of one chunk of partials (multiple of 128)
 };
 
@@ -81,7 +87,33 @@ struct StatsRow {
     int i1 = 0x7fffffff;
     int bump_col = -1;
     float bump_v = 0.f;
+    float best = -INFINITY;       // Gumbel-max draw: largest perturbed score so far and its token
+    int best_i = 0x7fffffff;
+    unsigned long long key = 0;   // start state of this row's random stream
 };
+
+// splitmix64 output function (Steele, Lea, Flood 2014); output number n of the stream with start state k is
+// mix64(k + n * 0x9E3779B97F4A7C15).
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// Per-row set-up of the LM-head epilogue: planted bump and, when sampling, the key of the row's stream
+// (seed, step and flat canvas position mixed together).
+__device__ __forceinline__ void stats_row_init(const GemmParams& p, int row, StatsRow& st) {
+    if (row >= *p.d_R) return;
+    const int flat = p.rows[row];
+    if (p.bump_id != nullptr) {
+        st.bump_col = p.bump_id[flat];
+        st.bump_v = p.bump_val[flat];
+    }
+    if (p.inv_temperature > 0.f) {
+        const unsigned long long step = (unsigned long long)(p.d_step ? *p.d_step : p.step_value);
+        st.key = mix64(p.sample_seed ^ (step << 40) ^ (unsigned long long)flat);
+    }
+}
 
 // Epilogue of one 128 x BN accumulator tile: the calling thread owns output row `row` (TMEM lane) and reads
 // it 32 columns at a time from tensor memory at `t_acc`.  Shared by the one-CTA and the CTA-pair kernels.
@@ -246,6 +278,19 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
             if (col0 + 32 > p.N) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = (col0 + j < p.N) ? v[j] : -INFINITY;
+            }
+            if (p.inv_temperature > 0.f) {
+                // Gumbel-max: argmax_v (l_v / T - ln(-ln u_v)), u_v from 23 bits of the row's counter stream
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const unsigned long long z = mix64(st.key + (unsigned long long)(col0 + j + 1) * 0x9E3779B97F4A7C15ull);
+                    const float u = ((float)(unsigned)(z >> 41) + 0.5f) * (1.f / 8388608.f);
+                    const float score = fmaf(v[j], p.inv_temperature, -logf(-logf(u)));
+                    if (score > st.best) {               // strict: the lowest token id wins ties
+                        st.best = score;
+                        st.best_i = col0 + j;
+                    }
+                }
             }
             float cm = v[0];
 #pragma unroll
@@ -424,15 +469,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         uint32_t acc_phase = 0;
         int m_blk, n_blk;
         StatsRow st;
-        if (EPI == EPI_STATS && total_tiles > 0) {
-            int R = *p.d_R;
-            int row = m_blk0 * kBM + row_in_tile;
-            if (row < R && p.bump_id != nullptr) {
-                int flat = p.rows[row];
-                st.bump_col = p.bump_id[flat];
-                st.bump_v = p.bump_val[flat];
-            }
-        }
+        if (EPI == EPI_STATS && total_tiles > 0) stats_row_init(p, m_blk0 * kBM + row_in_tile, st);
         bool ok = true;
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
@@ -445,8 +482,9 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
         if (EPI == EPI_STATS && ok && total_tiles > 0) {
-            p.partials[(size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile] =
-                make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
+            const size_t slot = (size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile;
+            p.partials[slot] = make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
+            if (p.inv_temperature > 0.f) p.partials2[slot] = make_float2(st.best, __int_as_float(st.best_i));
         }
     }
 

@@ -171,14 +171,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         uint32_t acc_phase = 0;
         int m_blk, n_blk;
         StatsRow st;
-        if (EPI == EPI_STATS && total_tiles > 0) {
-            const int row = m_blk0 * kBM + row_in_tile;
-            if (row < *p.d_R && p.bump_id != nullptr) {
-                const int flat = p.rows[row];
-                st.bump_col = p.bump_id[flat];
-                st.bump_v = p.bump_val[flat];
-            }
-        }
+        if (EPI == EPI_STATS && total_tiles > 0) stats_row_init(p, m_blk0 * kBM + row_in_tile, st);
         bool ok = true;
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
@@ -191,8 +184,9 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
         if (EPI == EPI_STATS && ok && total_tiles > 0 && stats_row_block_valid) {
-            p.partials[(size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile] =
-                make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
+            const size_t slot = (size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile;
+            p.partials[slot] = make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
+            if (p.inv_temperature > 0.f) p.partials2[slot] = make_float2(st.best, __int_as_float(st.best_i));
         }
     }
 

@@ -258,7 +258,9 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
                                                           int n_vt, int pair_mode, const int32_t* __restrict__ rows,
                                                           const int32_t* __restrict__ d_R, float* __restrict__ top1,
                                                           float* __restrict__ top2, float* __restrict__ sumexp,
-                                                          int32_t* __restrict__ argmax) {
+                                                          int32_t* __restrict__ argmax,
+                                                          const float2* __restrict__ partials2,
+                                                          int32_t* __restrict__ sampled) {
     grid_launch_dependents();
     grid_dependency_wait();
     const int R = *d_R;
@@ -281,6 +283,23 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
         u.S = __shfl_xor_sync(0xffffffffu, t.S, o);
         u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
         t = merge_tuples(t, u);
+    }
+    if (partials2) {
+        // the Gumbel-max draw: largest perturbed score over the chunks, the lower token id on a tie
+        float best = -INFINITY;
+        int best_i = 0x7fffffff;
+        for (int c = lane; c < n_ch; c += 32) {
+            const float2 v = partials2[(size_t)c * R_pad + r];
+            const int vi = __float_as_int(v.y);
+            if (v.x > best || (v.x == best && vi < best_i)) { best = v.x; best_i = vi; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+            if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
+        }
+        if (lane == 0) sampled[rows[r]] = best_i;
     }
     if (lane == 0) {
         const int flat = rows[r];

@@ -283,6 +283,8 @@ struct jot_model {
     __nv_bfloat16 *h, *a, *qkv, *vt, *attn, *act, *hsel;
     int32_t *rows, *rows_out, *seq_map;
     float4* partials;
+    float2* partials2;
+    int32_t* g_sampled;
     float* splitk;
     int R_cap;
     int32_t* canvas;      // generate: tokens [max_batch * max_seq]
@@ -336,7 +338,7 @@ struct ProfScope {
 };
 
 struct Layout {
-    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, rows_out, seq_map, partials, splitk, canvas, top1, top2, sumexp, argmax, state, params,
+    size_t ctrl, rope, h, a, qkv, vt, attn, act, hsel, rows, rows_out, seq_map, partials, partials2, sampled, splitk, canvas, top1, top2, sumexp, argmax, state, params,
         total;
 };
 
@@ -377,6 +379,8 @@ Layout make_layout(const jot_model_config* c, int max_batch, int max_seq) {
     l.rows_out = take(R_cap * 4);
     l.seq_map = take((size_t)max_batch * 4);
     l.partials = take((size_t)256 * R_cap * sizeof(float4));   // up to 256 vocabulary chunks
+    l.partials2 = take((size_t)256 * R_cap * sizeof(float2));
+    l.sampled = take(M * 4);
     l.splitk = take(kSplitKBytes);
     l.canvas = take(M * 4);
     l.top1 = take(M * 4);
@@ -478,14 +482,30 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
 }
 
 // hsel (active rows, already gathered) -> merged statistics scattered to the [B, L] outputs
+// Sampling-based finalisation of the head: temperature > 0 turns it on; the step index comes from the
+// device counter when d_step is given (generate loop), else from step_value.
+struct HeadSampling {
+    float temperature = 0.f;
+    unsigned long long seed = 0;
+    const int32_t* d_step = nullptr;
+    int step_value = 0;
+    int32_t* sampled = nullptr;      // [B, L] output
+};
+
 int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, const float* bump_val, float* top1,
-                      float* top2, float* sumexp, int32_t* argmax, int M, cudaStream_t st) {
+                      float* top2, float* sumexp, int32_t* argmax, int M, cudaStream_t st,
+                      const HeadSampling* hs = nullptr) {
     const jot_model_config& c = m->cfg;
     GemmParams p{};
     p.M = m->R_cap; p.N = c.vocab; p.K = c.d_model; p.status = m->ctrl;
     p.d_R = m->ctrl + 1; p.rows = m->rows_out; p.bump_id = bump_id; p.bump_val = bump_val;
     p.mask_col = exclude_mask ? c.mask_id : -1;
     p.partials = m->partials; p.R_pad = m->R_cap;
+    const bool sampling = hs && hs->temperature > 0.f;
+    if (sampling) {
+        p.inv_temperature = 1.f / hs->temperature; p.sample_seed = hs->seed; p.d_step = hs->d_step;
+        p.step_value = hs->step_value; p.partials2 = m->partials2;
+    }
     // few active rows: the head streams W once and is bandwidth bound -> narrow tiles balance the SMs best;
     // many rows: CTA pairs (256 x 256 tiles) halve the W bytes each SM takes in
     const int mode = (M <= 128) ? 0 : (M <= 256 ? 1 : 2);
@@ -506,7 +526,8 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     const int n_vt = (c.vocab + bn - 1) / bn;
     ProfScope ps(m, JOT_PROF_MERGE, st);
     launch_k(merge_stats_kernel, dim3((M + 3) / 4), dim3(128), 0, st, m->partials, m->R_cap, grid, n_vt, mode == 2 ? 1 : 0,
-             m->rows_out, m->ctrl + 1, top1, top2, sumexp, argmax);
+             m->rows_out, m->ctrl + 1, top1, top2, sumexp, argmax, sampling ? m->partials2 : nullptr,
+             sampling ? hs->sampled : nullptr);
     return launch_check();
 }
 
@@ -539,6 +560,17 @@ __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_b
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
 }
 
+// public sampling descriptor -> the head's; temperature <= 0 (or no descriptor) means argmax only
+int head_sampling_from(const jot_sampling* sp, int32_t* d_sampled, HeadSampling* hs) {
+    if (!sp || !(sp->temperature > 0.f)) return JOT_OK;
+    if (!d_sampled || sp->step < 0) return JOT_ERR_ARG;
+    hs->temperature = sp->temperature;
+    hs->seed = sp->seed;
+    hs->step_value = sp->step;
+    hs->sampled = d_sampled;
+    return JOT_OK;
+}
+
 int check_step_args(const jot_model* m, const void* tokens, int B, int L, int blk_lo, int blk_hi, const void* bump_id,
                     const void* bump_val, const void* o1, const void* o2, const void* o3, const void* o4) {
     if (!m || !tokens || !o1 || !o2 || !o3 || !o4) return JOT_ERR_ARG;
@@ -564,7 +596,11 @@ int launch_accept(const AcceptArgs& a, cudaStream_t st) {
     return launch_check();
 }
 
-bool params_ok(const jot_params* p) { return p && p->D >= 1 && p->D <= kMaxD; }
+bool params_ok(const jot_params* p) {
+    if (!p || p->D < 1 || p->D > kMaxD) return false;
+    if (p->gate == JOT_GATE_MAXPROB) return p->prob_threshold > 0.f && p->prob_threshold <= 1.f;
+    return p->gate == JOT_GATE_RATIO;
+}
 
 }  // namespace
 
@@ -630,6 +666,8 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
     m->rows_out = (int32_t*)(base + lay.rows_out);
     m->seq_map = (int32_t*)(base + lay.seq_map);
     m->partials = (float4*)(base + lay.partials);
+    m->partials2 = (float2*)(base + lay.partials2);
+    m->g_sampled = (int32_t*)(base + lay.sampled);
     m->splitk = (float*)(base + lay.splitk);
     m->R_cap = (int)align_up((size_t)max_batch * max_seq, 128);
     m->canvas = (int32_t*)(base + lay.canvas);
@@ -698,9 +736,12 @@ int jot_free_model(jot_model* m) {
 
 int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi,
                       int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val, float* d_top1,
-                      float* d_top2, float* d_sumexp, int32_t* d_argmax, void* stream) {
+                      float* d_top2, float* d_sumexp, int32_t* d_argmax, const jot_sampling* sampling,
+                      int32_t* d_sampled, void* stream) {
     JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
     if (!d_hidden) return JOT_ERR_ARG;
+    HeadSampling hs;
+    JOT_TRY(head_sampling_from(sampling, d_sampled, &hs));
     cudaStream_t st = (cudaStream_t)stream;
     JOT_TRY(encode_activation_maps(m, B, L));
     {
@@ -713,14 +754,16 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
         JOT_TRY(launch_check());
     }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
-                              B * (blk_hi - blk_lo), st));
+                              B * (blk_hi - blk_lo), st, &hs));
     return read_status(m, st);
 }
 
 int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi, int exclude_mask_token,
                      const int32_t* d_bump_id, const float* d_bump_val, float* d_top1, float* d_top2, float* d_sumexp,
-                     int32_t* d_argmax, void* stream) {
+                     int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled, void* stream) {
     JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
+    HeadSampling hs;
+    JOT_TRY(head_sampling_from(sampling, d_sampled, &hs));
     cudaStream_t st = (cudaStream_t)stream;
     JOT_TRY(forward_body(m, d_tokens, B, L, st));
     {
@@ -733,7 +776,7 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
         JOT_TRY(launch_check());
     }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
-                              B * (blk_hi - blk_lo), st));
+                              B * (blk_hi - blk_lo), st, &hs));
     return read_status(m, st);
 }
 
@@ -748,7 +791,7 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
     cudaStream_t st = (cudaStream_t)stream;
     AcceptArgs a{};
     a.uniform = AcceptParamsDev{params->tau_max, params->tau_min, params->gamma, params->D, params->eps,
-                                params->schedule_after_exit};
+                                params->schedule_after_exit, params->gate, params->prob_threshold};
     a.params = nullptr;
     a.mask_id = mask_id; a.tokens = d_tokens; a.B = B; a.L = L;
     a.blk_lo = blk_lo; a.blk_hi = blk_hi; a.k_transfer = k_transfer;
@@ -794,6 +837,17 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         if (!*finished) B_act = w[2];
         return JOT_OK;
     };
+    // sampling-based finalisation: the step index lives on the device (advanced by the acceptance kernel), so a
+    // captured step can be replayed unchanged
+    const bool sampling = gen->temperature > 0.f;
+    HeadSampling hs;
+    if (sampling) {
+        hs.temperature = gen->temperature;
+        hs.seed = ((unsigned long long)gen->seed_hi << 32) | gen->seed_lo;
+        hs.d_step = m->ctrl + 4;
+        hs.sampled = m->g_sampled;
+    }
+    JOT_CUDA(cudaMemsetAsync(m->ctrl + 4, 0, 4, st));
     // everything one step enqueues, ending with the copy of the control words to the pinned slot it & 1
     auto enqueue_step = [&](int it, int Bf, const int32_t* seq_map) -> int {
         JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
@@ -813,11 +867,13 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
             JOT_TRY(launch_check());
         }
         JOT_TRY(lm_head_from_hsel(m, gen->exclude_mask_token, d_bump_id, d_bump_val, m->g_top1, m->g_top2, m->g_sumexp,
-                                  m->g_argmax, Bf * gen->block_len, st));
+                                  m->g_argmax, Bf * gen->block_len, st, &hs));
         AcceptArgs a{};
         a.params = m->params_dev; a.per_seq_params = per_seq_params ? 1 : 0;
         a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
-        a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp; a.argmax = m->g_argmax;
+        a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp;
+        a.argmax = sampling ? m->g_sampled : m->g_argmax;       // the token a finalised position receives
+        a.step_counter = m->ctrl + 4;
         a.step_index = it + 1;                       // only reaches the optional exit-step output, unused here
         a.state = m->state; a.P = P; a.block_len = gen->block_len; a.n_blocks = nb; a.steps_per_block = Tb;
         a.n_unfinished = m->ctrl + 2;
@@ -888,11 +944,11 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         return rc;
     }
     JOT_CUDA(cudaMemcpyAsync(d_out_tokens, m->canvas, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
-    SeqState* hs = reinterpret_cast<SeqState*>(m->h_pinned + 16);
-    JOT_CUDA(cudaMemcpyAsync(hs, m->state, (size_t)B * sizeof(SeqState), cudaMemcpyDeviceToHost, st));
+    SeqState* host_state = reinterpret_cast<SeqState*>(m->h_pinned + 16);
+    JOT_CUDA(cudaMemcpyAsync(host_state, m->state, (size_t)B * sizeof(SeqState), cudaMemcpyDeviceToHost, st));
     JOT_CUDA(cudaStreamSynchronize(st));
     release_graphs();
-    for (int b = 0; b < B; ++b) h_steps_used[b] = hs[b].steps_used;
+    for (int b = 0; b < B; ++b) h_steps_used[b] = host_state[b].steps_used;
     if (h_forward_passes) *h_forward_passes = passes;
     return JOT_OK;
 }

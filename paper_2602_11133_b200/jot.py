@@ -37,13 +37,18 @@ class JotError(RuntimeError):
         super().__init__(f"{where}: {msg} (status {status}, cuda error {cuda})")
 
 
+GATE_RATIO, GATE_MAXPROB = 0, 1
+
+
 class Params(C.Structure):
     """tau_max, tau_min, gamma, D of Algorithm 1; eps of Eq. 4."""
     _fields_ = [("tau_max", C.c_float), ("tau_min", C.c_float), ("gamma", C.c_float), ("D", C.c_int32),
-                ("eps", C.c_float), ("schedule_after_exit", C.c_int32)]
+                ("eps", C.c_float), ("schedule_after_exit", C.c_int32), ("gate", C.c_int32),
+                ("prob_threshold", C.c_float)]
 
-    def __init__(self, tau_max=90.0, tau_min=1.0, gamma=0.5, D=8, eps=1e-12, schedule_after_exit=0):
-        super().__init__(tau_max, tau_min, gamma, D, eps, schedule_after_exit)
+    def __init__(self, tau_max=90.0, tau_min=1.0, gamma=0.5, D=8, eps=1e-12, schedule_after_exit=0, gate=0,
+                 prob_threshold=0.9):
+        super().__init__(tau_max, tau_min, gamma, D, eps, schedule_after_exit, gate, prob_threshold)
 
 
 class ModelConfig(C.Structure):
@@ -59,9 +64,15 @@ class _Weights(C.Structure):
                 ("w_down", C.POINTER(C.c_void_p))]
 
 
+class Sampling(C.Structure):
+    """Sampling-based finalisation: temperature > 0 draws each active row's token from softmax(l / T)."""
+    _fields_ = [("temperature", C.c_float), ("seed", C.c_uint64), ("step", C.c_int32)]
+
+
 class GenConfig(C.Structure):
     _fields_ = [("gen_len", C.c_int32), ("steps", C.c_int32), ("block_len", C.c_int32),
-                ("exclude_mask_token", C.c_int32), ("compact_finished", C.c_int32), ("use_cuda_graph", C.c_int32)]
+                ("exclude_mask_token", C.c_int32), ("compact_finished", C.c_int32), ("use_cuda_graph", C.c_int32),
+                ("temperature", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
 
 
 _LIB = None
@@ -83,7 +94,7 @@ def _lib():
                                        C.c_size_t, C.POINTER(C.c_void_p)]
         lib.jot_free_model.argtypes = [C.c_void_p]
         step_args = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
-                     C.c_void_p, C.c_void_p, C.c_void_p]
+                     C.c_void_p, C.c_void_p, C.POINTER(Sampling), C.c_void_p, C.c_void_p]
         lib.jot_denoise_step.argtypes = [C.c_void_p, C.c_void_p] + step_args
         lib.jot_lm_head_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + step_args
         lib.jot_accept_freeze.argtypes = [C.POINTER(Params), C.c_int, C.c_int32, C.c_void_p, C.c_int, C.c_int, C.c_int,
@@ -121,6 +132,15 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+def _sampling_args(sampling, out, B, L, device):
+    """(pointer to the descriptor or None, device pointer of the sampled-token array or None)."""
+    if sampling is None or not sampling.temperature > 0:
+        return None, None
+    if out.sampled is None:
+        out.sampled = torch.zeros(B, L, dtype=torch.int32, device=device)
+    return C.byref(sampling), _ptr(out.sampled, torch.int32, "sampled")
+
+
 def launch_count() -> int:
     return int(_lib().jot_launch_count())
 
@@ -132,6 +152,7 @@ class Stats:
     top2: torch.Tensor
     sumexp: torch.Tensor
     argmax: torch.Tensor
+    sampled: Optional[torch.Tensor] = None      # [B, L] int32, written when sampling is on
 
     @staticmethod
     def empty(B: int, L: int, device) -> "Stats":
@@ -194,35 +215,41 @@ class Model:
     # ---- one step -------------------------------------------------------------------------------
     def denoise_step(self, tokens: torch.Tensor, blk_lo: int, blk_hi: int, out: Optional[Stats] = None,
                      exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
-                     bump_val: Optional[torch.Tensor] = None) -> Stats:
+                     bump_val: Optional[torch.Tensor] = None, sampling: Optional[Sampling] = None) -> Stats:
         B, L = tokens.shape
         out = out or Stats.empty(B, L, tokens.device)
+        sp, d_sampled = _sampling_args(sampling, out, B, L, tokens.device)
         _check(_lib().jot_denoise_step(self.handle, _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo, blk_hi,
                                        int(exclude_mask_token), _ptr(bump_id, torch.int32, "bump_id"),
                                        _ptr(bump_val, torch.float32, "bump_val"), out.top1.data_ptr(),
-                                       out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), _stream()),
+                                       out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), sp,
+                                       d_sampled, _stream()),
                "jot_denoise_step")
         return out
 
     def lm_head_stats(self, hidden: torch.Tensor, tokens: torch.Tensor, blk_lo: int, blk_hi: int,
                       out: Optional[Stats] = None, exclude_mask_token: bool = True,
-                      bump_id: Optional[torch.Tensor] = None, bump_val: Optional[torch.Tensor] = None) -> Stats:
+                      bump_id: Optional[torch.Tensor] = None, bump_val: Optional[torch.Tensor] = None,
+                      sampling: Optional[Sampling] = None) -> Stats:
         B, L = tokens.shape
         if hidden.shape != (B * L, self.cfg.d_model):
             raise ValueError("hidden must be [B*L, d_model]")
         out = out or Stats.empty(B, L, tokens.device)
+        sp, d_sampled = _sampling_args(sampling, out, B, L, tokens.device)
         _check(_lib().jot_lm_head_stats(self.handle, _ptr(hidden, torch.bfloat16, "hidden"),
                                         _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo, blk_hi,
                                         int(exclude_mask_token), _ptr(bump_id, torch.int32, "bump_id"),
                                         _ptr(bump_val, torch.float32, "bump_val"), out.top1.data_ptr(),
-                                        out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), _stream()),
+                                        out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), sp,
+                                        d_sampled, _stream()),
                "jot_lm_head_stats")
         return out
 
     # ---- Algorithm 1 ----------------------------------------------------------------------------
     def generate(self, prompt: torch.Tensor, gen_len: int, steps: int, params, block_len: Optional[int] = None,
                  exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
-                 bump_val: Optional[torch.Tensor] = None, compact_finished: bool = True, use_cuda_graph: bool = False):
+                 bump_val: Optional[torch.Tensor] = None, compact_finished: bool = True, use_cuda_graph: bool = False,
+                 temperature: float = 0.0, seed: int = 0):
         """Returns (tokens [B, P+gen_len] int32 on device, steps_used list[int], forward_passes int)."""
         B, P = prompt.shape
         per_seq = isinstance(params, (list, tuple))
@@ -233,7 +260,7 @@ class Model:
         else:
             parr = (Params * 1)(params)
         gen = GenConfig(gen_len, steps, block_len or gen_len, int(exclude_mask_token), int(compact_finished),
-                        int(use_cuda_graph))
+                        int(use_cuda_graph), float(temperature), seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
         out = torch.empty(B, P + gen_len, dtype=torch.int32, device=prompt.device)
         used = (C.c_int32 * B)()
         passes = C.c_int32(0)

@@ -243,3 +243,108 @@ def test_lm_head_mask_token_and_ties(jot):
     model.lm_head_stats(hidden.cuda(), tokens.cuda(), 0, L, out=out)
     assert (out.sumexp == 1.0).all()
     model.close()
+
+
+# ---------------------------------------------------------------- sampling-based finalisation (Section 4.1)
+@pytest.mark.parametrize("B,P,G,d,V,T", [
+    (1, 32, 64, 256, 4096, 1.0),          # one narrow-tile chunk schedule
+    (2, 40, 200, 512, 5000, 0.7),         # ragged vocabulary tail, two row blocks
+    (8, 128, 256, 1024, 12800, 1.3),      # CTA-pair path
+])
+def test_lm_head_sampled_tokens_match_oracle(jot, B, P, G, d, V, T):
+    """The token drawn in the head's epilogue is the oracle's Gumbel-max draw from the same counter stream,
+    row by row; the unperturbed statistics do not depend on whether sampling is on."""
+    mask_id = V - 7
+    seed, step = 0x1234_5678_9ABC_DEF1, 5
+    case = inputs.lm_head_case(4, B, P, G, d, V, mask_id, device="cuda")
+    model = lm_head_model(jot, d, V, mask_id, case.w, B, P + G)
+    L = P + G
+    plain = model.lm_head_stats(case.hidden, case.tokens, P, L, bump_id=case.bump_id, bump_val=case.bump_val)
+    st = model.lm_head_stats(case.hidden, case.tokens, P, L, bump_id=case.bump_id, bump_val=case.bump_val,
+                             sampling=jot.Sampling(T, seed, step))
+    torch.cuda.synchronize()
+    for a, b in ((plain.top1, st.top1), (plain.top2, st.top2), (plain.sumexp, st.sumexp), (plain.argmax, st.argmax)):
+        assert torch.equal(a, b)
+    tok = case.tokens.cpu()
+    rows = [(b, i) for b in range(B) for i in range(P, L) if int(tok[b, i]) == mask_id]
+    if len(rows) > 160:                     # the oracle's draw costs a pass over V per row
+        rows = rows[:40] + rows[len(rows) // 2 - 40:len(rows) // 2 + 40] + rows[-40:]
+    flat = torch.tensor([b * L + i for b, i in rows])
+    logits = mo.lm_head_logits(case.hidden.cpu()[flat], case.w.cpu(), case.bump_id.cpu().view(-1)[flat],
+                               case.bump_val.cpu().view(-1)[flat]).numpy()
+    got = st.sampled.cpu().view(-1)[flat].tolist()
+    am = st.argmax.cpu().view(-1)[flat].tolist()
+    near = differs_from_argmax = 0
+    for r, f in enumerate(flat.tolist()):
+        want, gap = jo.sample_tokens_fast(logits[r], mask_id, T, seed, step, f)
+        scale = max(float(np.abs(np.delete(logits[r], mask_id)).max()), 1.0)
+        if gap < 2 * 1e-3 * scale / T:      # the two best perturbed scores are closer than the logit tolerance
+            near += 1
+            assert 0 <= got[r] < V and got[r] != mask_id
+            continue
+        assert got[r] == want, (r, f, got[r], want, gap)
+        differs_from_argmax += int(want != am[r])
+    assert near <= max(1, len(rows) // 50)
+    assert differs_from_argmax > len(rows) // 10          # a real draw, not the argmax in disguise
+    # another step index or seed gives another stream
+    st2 = model.lm_head_stats(case.hidden, case.tokens, P, L, bump_id=case.bump_id, bump_val=case.bump_val,
+                              sampling=jot.Sampling(T, seed, step + 1))
+    st3 = model.lm_head_stats(case.hidden, case.tokens, P, L, bump_id=case.bump_id, bump_val=case.bump_val,
+                              sampling=jot.Sampling(T, seed + 1, step))
+    a = st.sampled.view(-1)[flat.cuda()]
+    assert (st2.sampled.view(-1)[flat.cuda()] != a).float().mean() > 0.1
+    assert (st3.sampled.view(-1)[flat.cuda()] != a).float().mean() > 0.1
+    model.close()
+
+
+def test_lm_head_sampling_low_temperature_is_argmax(jot):
+    """T -> 0 makes the Gumbel term negligible: the draw equals the argmax wherever the top-2 gap is clear."""
+    d, V, B, P, G = 256, 4096, 2, 16, 112
+    mask_id = V - 7
+    case = inputs.lm_head_case(5, B, P, G, d, V, mask_id, device="cuda")
+    model = lm_head_model(jot, d, V, mask_id, case.w, B, P + G)
+    st = model.lm_head_stats(case.hidden, case.tokens, P, P + G, bump_id=case.bump_id, bump_val=case.bump_val,
+                             sampling=jot.Sampling(1e-3, 99, 0))
+    active = (case.tokens == mask_id)
+    active[:, :P] = False
+    clear = active & ((st.top1 - st.top2) > 0.05)           # Gumbel differences stay below ~30 * T
+    assert clear.sum() > 20 and torch.equal(st.sampled[clear], st.argmax[clear])
+    with pytest.raises(jot.JotError):
+        model.lm_head_stats(case.hidden, case.tokens, P, P + G, sampling=jot.Sampling(1.0, 1, -1))
+    model.close()
+
+
+@pytest.mark.parametrize("B,L,P,lo,hi,k", [(4, 384, 128, 128, 384, 1), (2, 1000, 10, 10, 1000, 7), (3, 704, 192, 224, 256, 1)])
+@pytest.mark.parametrize("pth", [0.5, 0.9])
+def test_accept_freeze_probability_gate_matches_oracle(jot, B, L, P, lo, hi, k, pth):
+    """The fixed gate p1 >= threshold that the paper contrasts the ratio test with (Section 2): same kernel,
+    same schedule and OR, no spatial modulation."""
+    V, mask_id = 5000, 4321
+    tokens, top1, top2, sumexp, argmax = random_accept_case(B * 77 + L, B, L, P, mask_id, V)
+    sumexp = (1.0 + (sumexp - 1.0) * 0.2).astype(np.float32)          # p1 spread on both sides of the gate
+    params = jo.JotParams(90, 1, 0.5, 8, gate="maxprob", prob_threshold=pth)
+    want, reps = oracle_accept_batch(torch.from_numpy(tokens), top1, top2, sumexp, argmax, params, mask_id, lo, hi, k)
+    d_tok = torch.from_numpy(tokens).cuda()
+    st = jot.Stats(*[torch.from_numpy(t).cuda() for t in (top1, top2, sumexp, argmax)])
+    reason = torch.zeros(B, L, dtype=torch.uint8, device="cuda")
+    jot.accept_freeze(jot.Params(90, 1, 0.5, 8, gate=jot.GATE_MAXPROB, prob_threshold=pth), mask_id, d_tok, lo, hi, k, st,
+                      exit_reason=reason)
+    got = d_tok.cpu()
+    n_exit = 0
+    for b in range(B):
+        nm = set(reps[b].near_margin)
+        n_exit += len(reps[b].exited)
+        for i in range(L):
+            if i in nm:
+                assert int(got[b, i]) in (mask_id, int(argmax[b, i]))
+            else:
+                assert int(got[b, i]) == int(want[b, i]), (b, i, 1.0 / sumexp[b, i])
+    assert n_exit > 0
+    # the ratio gate on the same statistics decides differently somewhere: the switch is really read
+    t2 = torch.from_numpy(tokens).cuda()
+    jot.accept_freeze(jot.Params(90, 1, 0.5, 8), mask_id, t2, lo, hi, k, st)
+    assert not torch.equal(t2, d_tok)
+    with pytest.raises(jot.JotError):
+        jot.accept_freeze(jot.Params(gate=2), mask_id, t2, lo, hi, k, st)
+    with pytest.raises(jot.JotError):
+        jot.accept_freeze(jot.Params(gate=jot.GATE_MAXPROB, prob_threshold=0.0), mask_id, t2, lo, hi, k, st)
