@@ -184,10 +184,25 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
  * sequence actually ran (step speed-up = steps / steps_used, Section 5.1); optional
  * h_forward_passes (host, one int) = batched forward passes executed.
  * d_bump_id / d_bump_val: as in jot_denoise_step, indexed [B, P + gen_len], fixed across steps.
+ * trace (nullable, any member nullable): what the paper's analysis plots are made of.  Device arrays,
+ * zeroed by the call and then written by the acceptance kernel:
+ *   d_exit_step [B, P + gen_len] int16: the sequence's own 1-based denoising step that finalised the
+ *     position (0: prompt); d_exit_reason, same shape, uint8: bit 0 early exit (Eq. 8), bit 1 transfer
+ *     schedule, both when both chose it;
+ *   d_mean_ratio [steps, B] float: mean confidence ratio r (Eq. 4) over the candidates the sequence had at
+ *     its s-th step (row s, 0-based; Appendix "Confidence Dynamics"); d_n_candidates, same shape, int32:
+ *     how many candidates that was.  Rows past a sequence's last step stay zero.
  * Synchronises `stream` once per step to read the loop condition. */
+typedef struct {
+    int16_t* d_exit_step;
+    uint8_t* d_exit_reason;
+    float* d_mean_ratio;
+    int32_t* d_n_candidates;
+} jot_trace;
 int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, const jot_gen_config* gen,
                  const int32_t* d_prompt, int B, int P, const int32_t* d_bump_id, const float* d_bump_val,
-                 int32_t* d_out_tokens, int32_t* h_steps_used, int32_t* h_forward_passes, void* stream);
+                 int32_t* d_out_tokens, int32_t* h_steps_used, int32_t* h_forward_passes, const jot_trace* trace,
+                 void* stream);
 
 /* C[M, N] (bf16) = A[M, K] (bf16) . W[N, K]^T (bf16) with fp32 accumulation on the tensor cores,
  * optionally + residual[M, N] (bf16, may alias C).  The projection every layer of the forward is made

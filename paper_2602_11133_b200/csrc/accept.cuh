@@ -52,6 +52,9 @@ struct AcceptArgs {
     int P, block_len, n_blocks, steps_per_block;
     int32_t* n_unfinished;           // device counter: += 1 per sequence that still has work (nullable)
     int32_t* step_counter;           // device counter of forward passes, advanced once per launch (nullable)
+    // generate mode, optional trace (Appendix "Confidence Dynamics"): row = the sequence's own 0-based step
+    float* mean_ratio;               // [steps, B]: mean of r over the step's candidates
+    int32_t* n_candidates;           // [steps, B]
 };
 
 // Dynamic shared memory: resolved bitmap words, candidate list, candidate sum-exp, candidate flags.
@@ -69,6 +72,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     __shared__ float gpow[kMaxD + 1];
     __shared__ int n_cand_sh, warp_counts[kAcceptThreads / 32], n_final_sh;
     __shared__ float inv_wmax;
+    __shared__ float ratio_sums[kAcceptThreads / 32];
 
     const AcceptParamsDev prm = a.params ? a.params[a.per_seq_params ? b : 0] : a.uniform;
     int32_t* x = a.tokens + (size_t)b * L;
@@ -130,6 +134,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     const int n_cand = n_cand_sh;
 
     // per candidate: ratio, threshold, early-exit decision
+    float r_sum = 0.f;
     for (int c = tid; c < n_cand; c += blockDim.x) {
         const int i = cand[c];
         const size_t gi = (size_t)b * L + i;
@@ -146,9 +151,15 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
         const float phi = fminf(1.f, w * inv_wmax);                        // Eq. 6
         const float tau = prm.tau_max - (prm.tau_max - prm.tau_min) * phi; // Eq. 7
         cand_S[c] = S;
+        r_sum += r;
         // Eq. 8; or the fixed probability gate the paper contrasts it with (p1 = 1/S, no spatial modulation)
         const bool exit_now = prm.gate == 1 ? (1.f / S >= prm.prob_threshold) : (r >= tau);
         cand_flag[c] = exit_now ? 1 : 0;
+    }
+    if (a.mean_ratio) {                                        // fixed-order tree: the same sum on every run
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) r_sum += __shfl_xor_sync(0xffffffffu, r_sum, o);
+        if ((tid & 31) == 0) ratio_sums[tid >> 5] = r_sum;
     }
     __syncthreads();
 
@@ -180,7 +191,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
             const size_t gi = (size_t)b * L + i;
             x[i] = a.argmax[gi];
             if (a.exit_reason) a.exit_reason[gi] = f;
-            if (a.exit_step) a.exit_step[gi] = (int16_t)a.step_index;
+            if (a.exit_step) a.exit_step[gi] = (int16_t)(a.state ? st.steps_used + 1 : a.step_index);
             ++my_final;
         }
     }
@@ -190,6 +201,12 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
         const int left = n_cand - n_final_sh;
         if (a.n_masked) a.n_masked[b] = left;
         if (a.state) {
+            if (n_cand > 0 && a.mean_ratio) {
+                float t = 0.f;
+                for (int w = 0; w < kAcceptThreads / 32; ++w) t += ratio_sums[w];
+                a.mean_ratio[(size_t)st.steps_used * a.B + b] = t / (float)n_cand;
+            }
+            if (n_cand > 0 && a.n_candidates) a.n_candidates[(size_t)st.steps_used * a.B + b] = n_cand;
             if (n_cand > 0) st.steps_used += 1;
             if (left == 0) { st.blk += 1; st.s = 0; } else { st.s += 1; }
             st.n_masked = left;

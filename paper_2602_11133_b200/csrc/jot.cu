@@ -804,7 +804,8 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
 
 int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, const jot_gen_config* gen,
                  const int32_t* d_prompt, int B, int P, const int32_t* d_bump_id, const float* d_bump_val,
-                 int32_t* d_out_tokens, int32_t* h_steps_used, int32_t* h_forward_passes, void* stream) {
+                 int32_t* d_out_tokens, int32_t* h_steps_used, int32_t* h_forward_passes, const jot_trace* trace,
+                 void* stream) {
     if (!m || !params || !gen || !d_out_tokens || !h_steps_used) return JOT_ERR_ARG;
     if ((d_bump_id == nullptr) != (d_bump_val == nullptr)) return JOT_ERR_ARG;
     if (B <= 0 || P < 0 || gen->gen_len <= 0 || gen->steps <= 0 || gen->block_len <= 0) return JOT_ERR_ARG;
@@ -823,6 +824,13 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     launch_k(init_canvas_kernel, dim3((B * L + 255) / 256), dim3(256), 0, st, d_prompt, m->canvas, B, P, gen->gen_len, m->cfg.mask_id,
                                                            m->state);
     JOT_TRY(launch_check());
+    if (trace) {                                     // positions and steps that never occur read as zero
+        if (trace->d_exit_step) JOT_CUDA(cudaMemsetAsync(trace->d_exit_step, 0, (size_t)B * L * sizeof(int16_t), st));
+        if (trace->d_exit_reason) JOT_CUDA(cudaMemsetAsync(trace->d_exit_reason, 0, (size_t)B * L, st));
+        if (trace->d_mean_ratio) JOT_CUDA(cudaMemsetAsync(trace->d_mean_ratio, 0, (size_t)gen->steps * B * sizeof(float), st));
+        if (trace->d_n_candidates)
+            JOT_CUDA(cudaMemsetAsync(trace->d_n_candidates, 0, (size_t)gen->steps * B * sizeof(int32_t), st));
+    }
     // The host runs one step ahead of what it knows: step `it` is enqueued before the outcome of step it-1 has
     // been read, so the GPU never idles while the host looks at the loop condition.  A step enqueued after the
     // last sequence finished finds nothing masked and changes nothing; it is not counted.
@@ -877,6 +885,10 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         a.step_index = it + 1;                       // only reaches the optional exit-step output, unused here
         a.state = m->state; a.P = P; a.block_len = gen->block_len; a.n_blocks = nb; a.steps_per_block = Tb;
         a.n_unfinished = m->ctrl + 2;
+        if (trace) {
+            a.exit_step = trace->d_exit_step; a.exit_reason = trace->d_exit_reason;
+            a.mean_ratio = trace->d_mean_ratio; a.n_candidates = trace->d_n_candidates;
+        }
         {
             ProfScope ps(m, JOT_PROF_ACCEPT, st);
             JOT_TRY(launch_accept(a, st));

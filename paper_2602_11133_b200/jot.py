@@ -75,6 +75,20 @@ class GenConfig(C.Structure):
                 ("temperature", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
 
 
+class _Trace(C.Structure):
+    _fields_ = [("exit_step", C.c_void_p), ("exit_reason", C.c_void_p), ("mean_ratio", C.c_void_p),
+                ("n_candidates", C.c_void_p)]
+
+
+@dataclasses.dataclass
+class Trace:
+    """Optional per-position / per-step record of a generation (device tensors)."""
+    exit_step: torch.Tensor        # [B, L] int16: 1-based step of the sequence that finalised the position
+    exit_reason: torch.Tensor      # [B, L] uint8: bit 0 early exit, bit 1 transfer schedule
+    mean_ratio: torch.Tensor       # [steps, B] float32: mean confidence ratio over the step's candidates
+    n_candidates: torch.Tensor     # [steps, B] int32
+
+
 _LIB = None
 
 
@@ -102,7 +116,7 @@ def _lib():
                                           C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         lib.jot_generate.argtypes = [C.c_void_p, C.POINTER(Params), C.c_int, C.POINTER(GenConfig), C.c_void_p, C.c_int,
                                      C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32),
-                                     C.POINTER(C.c_int32), C.c_void_p]
+                                     C.POINTER(C.c_int32), C.POINTER(_Trace), C.c_void_p]
         lib.jot_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                       C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         lib.jot_gemm_bf16_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
@@ -249,8 +263,9 @@ class Model:
     def generate(self, prompt: torch.Tensor, gen_len: int, steps: int, params, block_len: Optional[int] = None,
                  exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
                  bump_val: Optional[torch.Tensor] = None, compact_finished: bool = True, use_cuda_graph: bool = False,
-                 temperature: float = 0.0, seed: int = 0):
-        """Returns (tokens [B, P+gen_len] int32 on device, steps_used list[int], forward_passes int)."""
+                 temperature: float = 0.0, seed: int = 0, trace: bool = False):
+        """Returns (tokens [B, P+gen_len] int32 on device, steps_used list[int], forward_passes int), and a
+        Trace as a fourth element when trace is set."""
         B, P = prompt.shape
         per_seq = isinstance(params, (list, tuple))
         if per_seq:
@@ -264,9 +279,20 @@ class Model:
         out = torch.empty(B, P + gen_len, dtype=torch.int32, device=prompt.device)
         used = (C.c_int32 * B)()
         passes = C.c_int32(0)
+        tr, tr_arg = None, None
+        if trace:
+            dev = prompt.device
+            tr = Trace(torch.empty(B, P + gen_len, dtype=torch.int16, device=dev),
+                       torch.empty(B, P + gen_len, dtype=torch.uint8, device=dev),
+                       torch.empty(steps, B, dtype=torch.float32, device=dev),
+                       torch.empty(steps, B, dtype=torch.int32, device=dev))
+            tr_arg = C.byref(_Trace(tr.exit_step.data_ptr(), tr.exit_reason.data_ptr(), tr.mean_ratio.data_ptr(),
+                                    tr.n_candidates.data_ptr()))
         _check(_lib().jot_generate(self.handle, parr, int(per_seq), C.byref(gen), _ptr(prompt, torch.int32, "prompt"), B,
                                    P, _ptr(bump_id, torch.int32, "bump_id"), _ptr(bump_val, torch.float32, "bump_val"),
-                                   out.data_ptr(), used, C.byref(passes), _stream()), "jot_generate")
+                                   out.data_ptr(), used, C.byref(passes), tr_arg, _stream()), "jot_generate")
+        if trace:
+            return out, list(used), int(passes.value), tr
         return out, list(used), int(passes.value)
 
 

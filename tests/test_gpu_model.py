@@ -303,3 +303,58 @@ def test_sampled_generation_batch_graph_and_compaction(jot):
         assert same or tight, b
     print(f"sampled batch: {agree} of {B} sequences agree with the oracle token for token")
     model.close()
+
+
+def test_generation_trace_matches_oracle(jot):
+    """Exit step and exit reason of every position, and the mean confidence ratio of every step (the
+    quantities behind the paper's confidence-dynamics plots), against the oracle's trajectory."""
+    g = inputs.TINY
+    P, G, T, block_len = 32, 64, 64, 16
+    L = P + G
+    params = jo.LLADA_DEFAULT
+    w_cpu = inputs.model_weights(g, seed=0)
+    w_gpu = inputs.weights_to(w_cpu, "cuda")
+    prompt = inputs.prompt(0, 1, P, g.vocab, g.mask_id)
+    bump = inputs.logit_bump(9, 1, L, g.vocab, g.mask_id, hi=12.0)
+    tr = oracle_trajectory(g, w_cpu, prompt[0].tolist(), G, T, params, block_len, bump)
+    model = jot.Model(g, w_gpu, 2, L)
+    jp = jot.Params(params.tau_max, params.tau_min, params.gamma, params.D, params.eps)
+    ks = jo.transfer_counts(block_len, T // (G // block_len))
+    _, excused = replay_trajectory(jot, model, tr, params, g.mask_id, ks, bump)
+    out, used, passes, trace = model.generate(prompt.cuda(), G, T, jp, block_len, bump_id=bump[0].cuda(),
+                                              bump_val=bump[1].cuda(), trace=True)
+    es, er = trace.exit_step.cpu()[0].tolist(), trace.exit_reason.cpu()[0].tolist()
+    mr, nc = trace.mean_ratio.cpu()[:, 0].tolist(), trace.n_candidates.cpu()[:, 0].tolist()
+    # invariants that hold whatever the trajectory
+    assert all(e == 0 and r == 0 for e, r in zip(es[:P], er[:P]))
+    assert all(1 <= e <= used[0] and r in (1, 2, 3) for e, r in zip(es[P:], er[P:]))
+    assert all(n == 0 and m == 0.0 for n, m in zip(nc[used[0]:], mr[used[0]:])) and all(n > 0 for n in nc[:used[0]])
+    assert sum(1 for r in er[P:] if r & 2) >= used[0] - (G // block_len)      # the schedule reveals one per step
+    if excused == 0:
+        assert used[0] == tr.steps_used and out.cpu()[0].tolist() == tr.x
+        assert es == tr.exit_step
+        want_reason = [0] * L
+        for rep in tr.reports:
+            for i in rep.exited:
+                want_reason[i] |= 1
+            for i in rep.scheduled:
+                want_reason[i] |= 2
+        assert er == want_reason
+        for n, rep in enumerate(tr.reports):
+            assert nc[n] == len(rep.ratio)
+            want = sum(rep.ratio.values()) / len(rep.ratio)
+            # r = 1 / (exp(m2 - m1) + eps S): a logit error e changes ln r by up to ~e * r / (r + 1) per term
+            scale = 12.0                      # magnitude of the logits with the planted bump
+            assert abs(math.log(mr[n]) - math.log(want)) <= 2 * REL_TOL * scale, (n, mr[n], want)
+    print(f"trace: {used[0]} steps, {excused} excused; mean r first/last step {mr[0]:.3g} / {mr[used[0] - 1]:.3g}")
+    # the trace does not depend on batch neighbours, compaction or graph replay
+    prompt2 = torch.cat([prompt, inputs.prompt(3, 1, P, g.vocab, g.mask_id)]).cuda()
+    bid2 = torch.cat([bump[0], bump[0]]).cuda()
+    bval2 = torch.cat([bump[1], bump[1] * 0.5]).cuda()
+    for kw in (dict(), dict(compact_finished=False), dict(use_cuda_graph=True)):
+        o2, u2, _, t2 = model.generate(prompt2, G, T, jp, block_len, bump_id=bid2, bump_val=bval2, trace=True, **kw)
+        assert torch.equal(o2[0], out[0]) and u2[0] == used[0]
+        assert torch.equal(t2.exit_step[0], trace.exit_step[0]) and torch.equal(t2.exit_reason[0], trace.exit_reason[0])
+        assert torch.equal(t2.mean_ratio[:, 0], trace.mean_ratio[:, 0])
+        assert torch.equal(t2.n_candidates[:, 0], trace.n_candidates[:, 0])
+    model.close()
