@@ -20,6 +20,13 @@ path keeps in bf16 are rounded to bf16 here at the same named points, and nowher
 Pinned by tests against closed forms (RoPE rotation, attention row sums, permutation behaviour) and
 against an independent restatement built from torch.nn.functional routines; the float64/bf16
 contract itself is a reading of this build, not of the paper.
+
+Block-wise KV cache (hidden_states_cached, BlockCachedDenoiser): the paper names the cached decoder it
+composes with but does not define it; the reading taken is the published block-wise scheme with a cache on
+both sides of the block: refresh on entering a block, afterwards only the block's rows are recomputed.
+Pinned by: block = whole canvas reduces to the full pass; an unchanged canvas gives the full pass's rows;
+a token changed outside the block after the refresh is not seen; brute force with Python loops on a
+one-layer model.
 """
 from __future__ import annotations
 
@@ -40,20 +47,21 @@ def rmsnorm(h: torch.Tensor, gain: torch.Tensor, eps: float) -> torch.Tensor:
     return h * torch.rsqrt((h * h).mean(dim=-1, keepdim=True) + eps) * gain.to(F64)
 
 
-def rope(t: torch.Tensor, theta: float) -> torch.Tensor:
-    """t: [B, L, H, hd].  Rotate-half: pair (j, j + hd/2) turns by angle pos * theta^(-2j/hd)."""
-    B, L, H, hd = t.shape
+def rope(t: torch.Tensor, theta: float, pos0: int = 0) -> torch.Tensor:
+    """t: [B, n, H, hd], rows at canvas positions pos0 .. pos0+n-1.  Rotate-half: pair (j, j + hd/2) turns by
+    angle pos * theta^(-2j/hd)."""
+    B, n, H, hd = t.shape
     half = hd // 2
     inv = theta ** (-torch.arange(half, dtype=F64) * 2.0 / hd)
-    ang = torch.arange(L, dtype=F64)[:, None] * inv[None, :]          # [L, half]
+    ang = torch.arange(pos0, pos0 + n, dtype=F64)[:, None] * inv[None, :]   # [n, half]
     c, s = torch.cos(ang)[None, :, None, :], torch.sin(ang)[None, :, None, :]
     a, b = t[..., :half], t[..., half:]
     return torch.cat([a * c - b * s, b * c + a * s], dim=-1)
 
 
 def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, round_p: bool) -> torch.Tensor:
-    """q: [B, L, Hq, hd]; k, v: [B, L, Hkv, hd]; every query sees every key (no mask)."""
-    B, L, Hq, hd = q.shape
+    """q: [B, n, Hq, hd]; k, v: [B, L, Hkv, hd]; every query sees every key (no mask)."""
+    B, n, Hq, hd = q.shape
     group = Hq // k.shape[2]
     k = k.repeat_interleave(group, dim=2)
     v = v.repeat_interleave(group, dim=2)
@@ -64,30 +72,98 @@ def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, round_p: bool) 
     return o
 
 
+def layer(g, lw: Dict[str, torch.Tensor], h: torch.Tensor, ra: bool, pos0: int = 0, context=None):
+    """One transformer layer on rows h [B, n, d] that sit at canvas positions pos0 .. pos0+n-1.
+
+    context = None: the rows are the whole canvas and attend to each other.
+    context = (k, v), each [B, L, Hkv, hd], keys and values of the WHOLE canvas kept from an earlier pass
+    (block-wise KV cache): the rows' fresh k, v take the place of positions pos0 .. pos0+n-1 and the rows'
+    queries attend over all L positions; keys and values outside the rows stay as they were cached.
+    Returns (h_out [B, n, d], k [B, L, Hkv, hd], v [B, L, Hkv, hd]) with k, v as the attention used them."""
+    B, n, d = h.shape
+    nq, nkv, hd = g.n_q_heads, g.n_kv_heads, g.head_dim
+    a = _r(rmsnorm(h, lw["attn_norm"], g.rms_eps), ra)
+    qkv = _r(a @ lw["wqkv"].to(F64).T, ra)
+    q = qkv[..., : nq * hd].reshape(B, n, nq, hd)
+    k = qkv[..., nq * hd: (nq + nkv) * hd].reshape(B, n, nkv, hd)
+    v = qkv[..., (nq + nkv) * hd:].reshape(B, n, nkv, hd)
+    q = _r(rope(q, g.rope_theta, pos0), ra)
+    k = _r(rope(k, g.rope_theta, pos0), ra)
+    if context is not None:
+        k_all, v_all = context[0].clone(), context[1].clone()
+        k_all[:, pos0:pos0 + n] = k
+        v_all[:, pos0:pos0 + n] = v
+        k, v = k_all, v_all
+    o = _r(attention(q, k, v, ra), ra).reshape(B, n, nq * hd)
+    h = _r(h + o @ lw["wo"].to(F64).T, ra)
+    a = _r(rmsnorm(h, lw["mlp_norm"], g.rms_eps), ra)
+    gu = a @ lw["w_gate_up"].to(F64).T
+    gate, up = gu[..., : g.d_ff], gu[..., g.d_ff:]
+    act = _r(gate * torch.sigmoid(gate) * up, ra)
+    h = _r(h + act @ lw["w_down"].to(F64).T, ra)
+    return h, k, v
+
+
 def hidden_states(g, w: Dict[str, object], tokens: torch.Tensor, round_activations: bool = True,
-                  n_layers: Optional[int] = None) -> torch.Tensor:
-    """Final-normalised hidden states [B, L, d] (float64, bf16-valued when rounding is on)."""
+                  n_layers: Optional[int] = None, cache_out: Optional[list] = None) -> torch.Tensor:
+    """Final-normalised hidden states [B, L, d] (float64, bf16-valued when rounding is on).
+    cache_out, when a list, receives one (k, v) per layer: what a block-wise KV cache keeps of this pass."""
     ra = round_activations
-    B, L = tokens.shape
-    nq, nkv, hd, d = g.n_q_heads, g.n_kv_heads, g.head_dim, g.d_model
     h = w["embed"][tokens.long()].to(F64)                               # [B, L, d]
     layers = w["layers"] if n_layers is None else w["layers"][:n_layers]
     for lw in layers:
-        a = _r(rmsnorm(h, lw["attn_norm"], g.rms_eps), ra)
-        qkv = _r(a @ lw["wqkv"].to(F64).T, ra)
-        q = qkv[..., : nq * hd].reshape(B, L, nq, hd)
-        k = qkv[..., nq * hd: (nq + nkv) * hd].reshape(B, L, nkv, hd)
-        v = qkv[..., (nq + nkv) * hd:].reshape(B, L, nkv, hd)
-        q = _r(rope(q, g.rope_theta), ra)
-        k = _r(rope(k, g.rope_theta), ra)
-        o = _r(attention(q, k, v, ra), ra).reshape(B, L, nq * hd)
-        h = _r(h + o @ lw["wo"].to(F64).T, ra)
-        a = _r(rmsnorm(h, lw["mlp_norm"], g.rms_eps), ra)
-        gu = a @ lw["w_gate_up"].to(F64).T
-        gate, up = gu[..., : g.d_ff], gu[..., g.d_ff:]
-        act = _r(gate * torch.sigmoid(gate) * up, ra)
-        h = _r(h + act @ lw["w_down"].to(F64).T, ra)
+        h, k, v = layer(g, lw, h, ra)
+        if cache_out is not None:
+            cache_out.append((k, v))
     return _r(rmsnorm(h, w["final_norm"], g.rms_eps), ra)
+
+
+def hidden_states_cached(g, w: Dict[str, object], tokens: torch.Tensor, cache: list, lo: int, hi: int,
+                         round_activations: bool = True) -> torch.Tensor:
+    """Final-normalised hidden states [B, hi-lo, d] of canvas rows lo..hi-1 under a block-wise KV cache
+    (the block-wise cache JoT is composed with in Section 6.2, "Composability with KV-cache acceleration"): only these rows
+    go through the network; in every layer they attend over their own fresh keys / values and over the
+    cached keys / values of every position before AND after them.  `cache` is what hidden_states(...,
+    cache_out=) recorded on an earlier canvas; it is not modified."""
+    ra = round_activations
+    h = w["embed"][tokens[:, lo:hi].long()].to(F64)
+    assert len(cache) == len(w["layers"])
+    for lw, ctx in zip(w["layers"], cache):
+        h, _, _ = layer(g, lw, h, ra, pos0=lo, context=ctx)
+    return _r(rmsnorm(h, w["final_norm"], g.rms_eps), ra)
+
+
+class BlockCachedDenoiser:
+    """f_theta as a block-wise cached decoder sees it, for jot_oracle.generate (one sequence).
+
+    The first call that asks for rows of a block runs the full pass on the canvas as it is then, answers
+    from it, and keeps every layer's keys and values; later calls for the same block run only the block's
+    rows against that cache.  Entering another block refreshes the cache.  bump = (ids [L], values [L]) is
+    the planted logit bump of the synthetic workloads."""
+
+    def __init__(self, g, w, P: int, block_len: int, bump=None, round_activations: bool = True):
+        self.g, self.w, self.P, self.Lb, self.bump, self.ra = g, w, P, block_len, bump, round_activations
+        self.block, self.cache = None, None
+        self.full_passes = self.cached_passes = 0
+
+    def __call__(self, x, rows):
+        t = torch.tensor([list(x)], dtype=torch.int32)
+        blk = (rows[0] - self.P) // self.Lb
+        lo = self.P + blk * self.Lb
+        assert all(lo <= i < lo + self.Lb for i in rows)
+        if blk != self.block:
+            self.cache = []
+            h = hidden_states(self.g, self.w, t, self.ra, cache_out=self.cache)[0, lo:lo + self.Lb]
+            self.block = blk
+            self.full_passes += 1
+        else:
+            h = hidden_states_cached(self.g, self.w, t, self.cache, lo, lo + self.Lb, self.ra)[0]
+            self.cached_passes += 1
+        sel = torch.stack([h[i - lo] for i in rows])
+        idx = torch.tensor(rows)
+        l = lm_head_logits(sel, self.w["lm_head"], None if self.bump is None else self.bump[0][idx],
+                           None if self.bump is None else self.bump[1][idx])
+        return {i: l[r].numpy() for r, i in enumerate(rows)}
 
 
 def lm_head_logits(hidden_rows: torch.Tensor, w_lm: torch.Tensor,

@@ -2,6 +2,7 @@
 built from torch.nn.functional routines."""
 import math
 
+import numpy as np
 import pytest
 import torch
 import torch.nn.functional as F
@@ -160,3 +161,155 @@ def test_inputs_are_seeded_and_well_formed():
     assert 0.45 < frac < 0.55
     ids, val = inputs.logit_bump(0, 8, 384, 126464, 126336)
     assert (ids != 126336).all() and val.min() >= 0 and val.max() <= 12 and val.dtype == torch.float32
+
+
+# ---------------------------------------------------------------- block-wise KV cache
+def _tiny_case(seed=2, B=2, P=6, G=18):
+    g = inputs.ModelGeometry(2, 64, 2, 1, 32, 96, 128, 127, 10000.0)
+    w = inputs.model_weights(g, seed=seed)
+    tokens = inputs.partially_masked_canvas(seed, B, P, G, g.vocab, g.mask_id, 0.6)
+    return g, w, tokens
+
+
+def test_cached_pass_with_block_equal_to_canvas_is_the_full_pass():
+    g, w, tokens = _tiny_case()
+    cache = []
+    full = mo.hidden_states(g, w, tokens, cache_out=cache)
+    assert len(cache) == g.n_layers and cache[0][0].shape == (2, 24, g.n_kv_heads, g.head_dim)
+    # the cache's content is irrelevant when every position is recomputed
+    junk = [(torch.full_like(k, 7.0), torch.full_like(v, -3.0)) for k, v in cache]
+    got = mo.hidden_states_cached(g, w, tokens, junk, 0, tokens.shape[1])
+    assert torch.equal(got, full)
+
+
+@pytest.mark.parametrize("lo,hi", [(6, 12), (12, 24), (0, 6), (9, 10)])
+def test_cached_pass_on_an_unchanged_canvas_gives_the_full_pass_rows(lo, hi):
+    for ra in (True, False):
+        g, w, tokens = _tiny_case()
+        cache = []
+        full = mo.hidden_states(g, w, tokens, round_activations=ra, cache_out=cache)
+        got = mo.hidden_states_cached(g, w, tokens, cache, lo, hi, round_activations=ra)
+        assert got.shape == (2, hi - lo, g.d_model)
+        assert torch.allclose(got, full[:, lo:hi], rtol=0, atol=1e-12 if not ra else 0.0)
+
+
+def test_cache_is_stale_outside_the_block_and_fresh_inside():
+    g, w, tokens = _tiny_case()
+    lo, hi = 12, 18
+    cache = []
+    mo.hidden_states(g, w, tokens, cache_out=cache)
+    base = mo.hidden_states_cached(g, w, tokens, cache, lo, hi)
+    outside = tokens.clone()
+    outside[:, 3] = (outside[:, 3] + 5) % 100          # prefix token changes after the refresh
+    outside[:, 20] = (outside[:, 20] + 9) % 100        # and a suffix token
+    assert torch.equal(mo.hidden_states_cached(g, w, outside, cache, lo, hi), base)       # not seen
+    assert not torch.equal(mo.hidden_states(g, w, outside)[:, lo:hi], base)               # the full pass sees it
+    inside = tokens.clone()
+    inside[:, 14] = (inside[:, 14] + 11) % 100
+    got = mo.hidden_states_cached(g, w, inside, cache, lo, hi)
+    assert not torch.equal(got, base)                                                     # seen by the block's rows
+    # and it is an approximation of the full pass on the new canvas, not equal to it: positions outside the
+    # block would have reacted to the new token
+    full_new = mo.hidden_states(g, w, inside)[:, lo:hi]
+    diff = (got - full_new).abs().max().item()
+    assert 0 < diff < 0.5 * full_new.abs().max().item()
+    # the cache itself is never written
+    again = []
+    mo.hidden_states(g, w, tokens, cache_out=again)
+    assert all(torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) for a, b in zip(cache, again))
+
+
+def test_cached_layer_against_loops():
+    """One layer, one head, no rounding: attention of a block row written out with Python loops over keys,
+    taking fresh keys / values inside the block and the cached ones outside."""
+    g = inputs.ModelGeometry(1, 16, 1, 1, 16, 32, 64, 63, 10000.0)
+    w = inputs.model_weights(g, seed=4)
+    L, lo, hi = 10, 4, 7
+    old = inputs.partially_masked_canvas(4, 1, 2, L - 2, g.vocab, g.mask_id, 0.5)
+    new = old.clone()
+    new[0, 5] = 17
+    cache = []
+    mo.hidden_states(g, w, old, round_activations=False, cache_out=cache)
+    lw = w["layers"][0]
+    h_new = w["embed"][new.long()].double()[0]                                 # [L, d]
+    hd = g.head_dim
+
+    def qkv_row(h_row, pos):
+        a = h_row * (h_row.pow(2).mean() + g.rms_eps).rsqrt() * lw["attn_norm"].double()
+        z = lw["wqkv"].double() @ a
+        q, k, v = z[:hd], z[hd:2 * hd], z[2 * hd:]
+        def rot(t):
+            out = t.clone()
+            for j in range(hd // 2):
+                ang = pos * g.rope_theta ** (-2.0 * j / hd)
+                out[j] = t[j] * math.cos(ang) - t[j + hd // 2] * math.sin(ang)
+                out[j + hd // 2] = t[j + hd // 2] * math.cos(ang) + t[j] * math.sin(ang)
+            return out
+        return rot(q), rot(k), v
+
+    fresh = {i: qkv_row(h_new[i], i) for i in range(lo, hi)}
+    want = []
+    for i in range(lo, hi):
+        q = fresh[i][0]
+        scores, vals = [], []
+        for j in range(L):
+            k_j = fresh[j][1] if lo <= j < hi else cache[0][0][0, j, 0]
+            v_j = fresh[j][2] if lo <= j < hi else cache[0][1][0, j, 0]
+            scores.append(float(q @ k_j) / math.sqrt(hd))
+            vals.append(v_j)
+        mx = max(scores)
+        e = [math.exp(s - mx) for s in scores]
+        o = sum(ei * vj for ei, vj in zip(e, vals)) / sum(e)
+        h1 = h_new[i] + lw["wo"].double() @ o
+        a = h1 * (h1.pow(2).mean() + g.rms_eps).rsqrt() * lw["mlp_norm"].double()
+        gu = lw["w_gate_up"].double() @ a
+        gate, up = gu[:g.d_ff], gu[g.d_ff:]
+        h2 = h1 + lw["w_down"].double() @ (gate / (1 + torch.exp(-gate)) * up)
+        want.append(h2 * (h2.pow(2).mean() + g.rms_eps).rsqrt() * w["final_norm"].double())
+    got = mo.hidden_states_cached(g, w, new, cache, lo, hi, round_activations=False)[0]
+    assert torch.allclose(got, torch.stack(want), rtol=1e-10, atol=1e-12)
+
+
+def test_block_cached_denoiser_refreshes_on_block_change():
+    g, w, _ = _tiny_case()
+    P, G, Lb = 6, 18, 6
+    x = inputs.prompt(1, 1, P, g.vocab, g.mask_id)[0].tolist() + [g.mask_id] * G
+    den = mo.BlockCachedDenoiser(g, w, P, Lb)
+    first = den(x, [6, 7, 8, 9, 10, 11])
+    full = mo.logits(g, w, torch.tensor([x], dtype=torch.int32), rows=[(0, i) for i in range(6, 12)])
+    assert all(np.array_equal(first[i], full[r].numpy()) for r, i in enumerate(range(6, 12)))   # refresh = full pass
+    x[7] = 3
+    den(x, [6, 8, 9])
+    assert (den.full_passes, den.cached_passes) == (1, 1)
+    x[6] = x[8] = x[9] = x[10] = x[11] = 5
+    den(x, [12, 13])                                     # next block: refresh, again the full pass
+    assert (den.full_passes, den.cached_passes) == (2, 1)
+    full = mo.logits(g, w, torch.tensor([x], dtype=torch.int32), rows=[(0, 12), (0, 13)])
+    again = den(x, [12, 13])                             # same canvas, now through the cache: same rows
+    assert np.allclose(again[12], full[0].numpy(), rtol=0, atol=1e-9)
+    assert (den.full_passes, den.cached_passes) == (2, 2)
+
+
+def test_generation_under_the_block_cache():
+    """Algorithm 1 over the cached denoiser: one full pass per block, every other step recomputes the block
+    only; with a single block spanning the whole generation the first step equals the uncached run's."""
+    from oracle import jot_oracle as jo
+    g, w, _ = _tiny_case()
+    P, G, Lb, T = 6, 18, 6, 18
+    prompt = inputs.prompt(1, 1, P, g.vocab, g.mask_id)[0].tolist()
+    bump = inputs.logit_bump(2, 1, P + G, g.vocab, g.mask_id, hi=10.0)
+    bump = (bump[0][0], bump[1][0])
+    den = mo.BlockCachedDenoiser(g, w, P, Lb, bump)
+    tr = jo.generate(den, prompt, G, T, jo.JotParams(30, 1, 0.5, 4), g.mask_id, Lb)
+    assert all(t != g.mask_id for t in tr.x)
+    assert den.full_passes == G // Lb and den.full_passes + den.cached_passes == tr.steps_used
+    plain = mo.BlockCachedDenoiser(g, w, P, G, bump)          # one block: first step is the plain full pass
+    tr1 = jo.generate(plain, prompt, G, T, jo.JotParams(30, 1, 0.5, 4), g.mask_id, G)
+
+    def uncached(x, rows):
+        l = mo.logits(g, w, torch.tensor([x], dtype=torch.int32), rows=[(0, i) for i in rows])
+        for r, i in enumerate(rows):
+            l[r, int(bump[0][i])] += float(bump[1][i])
+        return {i: l[r].numpy() for r, i in enumerate(rows)}
+    tr2 = jo.generate(uncached, prompt, G, T, jo.JotParams(30, 1, 0.5, 4), g.mask_id, G)
+    assert tr1.canvases[1] == tr2.canvases[1]

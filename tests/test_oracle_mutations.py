@@ -166,16 +166,16 @@ def test_decision_pins_catch(name, monkeypatch):
 
 
 # ---------------------------------------------------------------- denoiser side
-def mut_rope_wrong_sign(t, theta):
-    out = ORIG_M["rope"](t, theta)
+def mut_rope_wrong_sign(t, theta, pos0=0):
+    out = ORIG_M["rope"](t, theta, pos0)
     half = t.shape[-1] // 2
     return torch.cat([out[..., :half], -out[..., half:]], dim=-1)
 
 
-def mut_rope_interleaved(t, theta):
+def mut_rope_interleaved(t, theta, pos0=0):
     B, L, H, hd = t.shape
     inv = theta ** (-torch.arange(hd // 2, dtype=torch.float64) * 2.0 / hd)
-    ang = torch.arange(L, dtype=torch.float64)[:, None] * inv[None, :]
+    ang = torch.arange(pos0, pos0 + L, dtype=torch.float64)[:, None] * inv[None, :]
     c, s = torch.cos(ang)[None, :, None, :], torch.sin(ang)[None, :, None, :]
     a, b = t[..., 0::2], t[..., 1::2]
     out = torch.empty_like(t)
@@ -218,7 +218,39 @@ def mut_lm_head_bump_everywhere(hidden_rows, w_lm, bump_id=None, bump_val=None):
     return l
 
 
-ORIG_M = {n: getattr(mo, n) for n in ("rope", "attention", "rmsnorm", "lm_head_logits")}
+def mut_rope_block_rows_start_at_zero(t, theta, pos0=0):
+    return ORIG_M["rope"](t, theta, 0)
+
+
+def mut_layer_cache_drops_the_suffix(g, lw, h, ra, pos0=0, context=None):
+    if context is not None:                       # a prefix-only cache: nothing after the block is attended to
+        end = pos0 + h.shape[1]
+        context = (context[0][:, :end], context[1][:, :end])
+    return ORIG_M["layer"](g, lw, h, ra, pos0, context)
+
+
+def mut_layer_cache_ignored(g, lw, h, ra, pos0=0, context=None):
+    return ORIG_M["layer"](g, lw, h, ra, pos0, None)      # the block attends only to itself
+
+
+ORIG_M = {n: getattr(mo, n) for n in ("rope", "attention", "rmsnorm", "lm_head_logits", "layer")}
+CACHE_PINS = [pins_m.test_cached_pass_with_block_equal_to_canvas_is_the_full_pass,
+              pins_m.test_cached_pass_on_an_unchanged_canvas_gives_the_full_pass_rows,
+              pins_m.test_cache_is_stale_outside_the_block_and_fresh_inside, pins_m.test_cached_layer_against_loops]
+CACHE_MUTATIONS = {
+    "cache: block rows rotated as if they sat at position 0": ("rope", mut_rope_block_rows_start_at_zero),
+    "cache: keys and values after the block dropped": ("layer", mut_layer_cache_drops_the_suffix),
+    "cache: context ignored": ("layer", mut_layer_cache_ignored),
+}
+
+
+@pytest.mark.parametrize("name", sorted(CACHE_MUTATIONS))
+def test_cache_pins_catch(name, monkeypatch):
+    assert not some_pin_fails(CACHE_PINS)
+    attr, fn = CACHE_MUTATIONS[name]
+    monkeypatch.setattr(mo, attr, fn)
+    assert some_pin_fails(CACHE_PINS), f"no pin noticed: {name}"
+
 
 MODEL_MUTATIONS = {
     "rope: rotation in the wrong direction on one half": ("rope", mut_rope_wrong_sign),
