@@ -95,6 +95,11 @@ typedef struct {
  * out of the candidate predictions.  compact_finished: the paper decodes one sequence at a time, where
  * early stopping ends the loop; in a batch the loop runs until the slowest sequence is done, and with this
  * flag the forward pass only covers the sequences still decoding (same tokens and step counts, fewer rows).
+ * kv_cache: the composition with a block-wise KV cache that Section 6.2 ("Composability with KV-cache
+ * acceleration") measures; see jot_denoise_step_cached for what a step then computes.  All sequences work on
+ * the same block and move on together once none of them has a masked position left in it (a sequence that
+ * is done with the block idles, its step count stands still); compact_finished and use_cuda_graph are
+ * ignored; the host reads the outcome of every step before it enqueues the next.
  * use_cuda_graph: the kernels of one step are captured on `stream` (which therefore must not already be
  * capturing) and replayed as one graph launch per step; pays off when a step is a few dozen short kernels. */
 typedef struct {
@@ -103,7 +108,9 @@ typedef struct {
     int32_t compact_finished;   /* != 0: sequences that have finished drop out of later forward passes */
     int32_t use_cuda_graph;     /* != 0: a step is captured into a CUDA graph once and replayed */
     float temperature;          /* > 0: finalised positions receive a sample from softmax(l / temperature) */
-    uint32_t seed_lo, seed_hi;  /* the 64-bit seed of jot_sampling; the step is the forward pass index */
+    uint32_t seed_lo, seed_hi;  /* the 64-bit seed of jot_sampling; a row's step is its sequence's own count of
+                                   denoising steps so far, so a draw does not depend on the rest of the batch */
+    int32_t kv_cache;           /* != 0: decode under the block-wise KV cache (needs jot_attach_kv_cache) */
 } jot_gen_config;
 
 /* Sampling-based finalisation (Section 4.1, "Early-Exit Decision": the finalised token may be drawn from
@@ -149,6 +156,27 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
                      float* d_top1_logit, float* d_top2_logit, float* d_sumexp, int32_t* d_argmax,
                      const jot_sampling* sampling /* nullable */, int32_t* d_sampled /* [B, L], with sampling */,
                      void* stream);
+
+/* Block-wise KV cache (Section 6.2, "Composability with KV-cache acceleration": JoT run inside a decoder that
+ * caches keys and values block by block).  The paper names that decoder without defining it; the scheme
+ * built here is the published one with a cache on both sides of the block:
+ *   refresh != 0  the whole canvas goes through the network exactly as in jot_denoise_step, and every
+ *                 layer's rotated keys and its values, for all L positions, stay in the attached cache;
+ *   refresh == 0  only rows [blk_lo, blk_hi) go through the network; in every layer their fresh keys and
+ *                 values replace the cache's entries for those positions and their queries attend over
+ *                 all L positions, the others as cached.  Needs an earlier refresh with the same B and L
+ *                 (else JOT_ERR_ARG).  Per step this costs (blk_hi - blk_lo) / L of the full pass's
+ *                 projections; its statistics are approximate wherever the canvas has changed outside
+ *                 the block since the refresh.
+ * The cache is caller-owned device memory of jot_kv_cache_bytes(cfg, max_batch, max_seq) bytes, 1 KiB
+ * aligned, attached with jot_attach_kv_cache (d_cache = NULL detaches) and borrowed until detached or the
+ * model is freed; attaching invalidates what was cached.  Outputs and options as in jot_denoise_step. */
+size_t jot_kv_cache_bytes(const jot_model_config* cfg, int max_batch, int max_seq);
+int jot_attach_kv_cache(jot_model* m, void* d_cache, size_t bytes);
+int jot_denoise_step_cached(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi,
+                            int refresh, int exclude_mask_token, const int32_t* d_bump_id,
+                            const float* d_bump_val, float* d_top1_logit, float* d_top2_logit, float* d_sumexp,
+                            int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled, void* stream);
 
 /* The LM head + statistics part of jot_denoise_step alone, on caller-supplied final hidden states
  * d_hidden [B*L, d] bf16 (already normalised).  Uses only lm_head, vocab, mask_id and d_model of

@@ -51,7 +51,8 @@ struct AcceptArgs {
     SeqState* state;                 // [B] nullable
     int P, block_len, n_blocks, steps_per_block;
     int32_t* n_unfinished;           // device counter: += 1 per sequence that still has work (nullable)
-    int32_t* step_counter;           // device counter of forward passes, advanced once per launch (nullable)
+    int lockstep;                    // generate mode under a block-wise KV cache: every sequence works on the block
+                                     // [blk_lo, blk_hi) with k_transfer; the host moves all of them on together
     // generate mode, optional trace (Appendix "Confidence Dynamics"): row = the sequence's own 0-based step
     float* mean_ratio;               // [steps, B]: mean of r over the step's candidates
     int32_t* n_candidates;           // [steps, B]
@@ -63,7 +64,6 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     grid_launch_dependents();
     grid_dependency_wait();
     const int L = a.L, b = blockIdx.x, tid = threadIdx.x;
-    if (a.step_counter && b == 0 && tid == 0) atomicAdd(a.step_counter, 1);
     const int n_words = (L + 31) / 32;
     uint32_t* res_bits = sh;                                   // [n_words + 2] resolved bitmap (padded)
     int* cand = reinterpret_cast<int*>(sh + n_words + 2);     // [L] candidate positions, ascending
@@ -79,8 +79,8 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
 
     int lo = a.blk_lo, hi = a.blk_hi, k = a.k_transfer;
     SeqState st = {0, 0, 0, 0};
-    if (a.state) {
-        st = a.state[b];
+    if (a.state) st = a.state[b];
+    if (a.state && !a.lockstep) {
         if (st.blk >= a.n_blocks) return;                      // finished sequence idles (uniform exit)
         lo = a.P + st.blk * a.block_len;
         hi = lo + a.block_len;
@@ -208,10 +208,15 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
             }
             if (n_cand > 0 && a.n_candidates) a.n_candidates[(size_t)st.steps_used * a.B + b] = n_cand;
             if (n_cand > 0) st.steps_used += 1;
-            if (left == 0) { st.blk += 1; st.s = 0; } else { st.s += 1; }
             st.n_masked = left;
-            a.state[b] = st;
-            if (a.n_unfinished && st.blk < a.n_blocks) atomicAdd(a.n_unfinished, 1);
+            if (a.lockstep) {                                  // the host advances the block for everyone
+                a.state[b] = st;
+                if (a.n_unfinished && left > 0) atomicAdd(a.n_unfinished, 1);
+            } else {
+                if (left == 0) { st.blk += 1; st.s = 0; } else { st.s += 1; }
+                a.state[b] = st;
+                if (a.n_unfinished && st.blk < a.n_blocks) atomicAdd(a.n_unfinished, 1);
+            }
         }
     }
 }

@@ -30,8 +30,11 @@ constexpr int kAttnSoftmaxThreads = 256;
 struct AttnParams {
     int B, L, nq, nkv;
     float scale_log2e;            // log2(e) / sqrt(hd)
-    __nv_bfloat16* out;           // [B*L, nq*hd]
+    __nv_bfloat16* out;           // [B*q_cnt, nq*hd]: row b * q_cnt + (q - q_lo)
     int32_t* status;
+    // queries are canvas positions q_lo .. q_lo + q_cnt - 1 of every sequence (the whole canvas: 0, L; one block
+    // of a block-wise KV cache: its rows only); keys and values are always all L positions
+    int q_lo, q_cnt;
 };
 
 template <int HD>
@@ -68,7 +71,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int L = p.L;
-    const int nkb = (L + 127) / 128, nqb = nkb;
+    const int nkb = (L + 127) / 128, nqb = (p.q_cnt + 127) / 128;
     const int group = p.nq / p.nkv;
     const int n_items = p.B * p.nq * nqb;
 
@@ -129,7 +132,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
                 mbar_arrive_expect_tx(&q_full, SM::Q_BYTES);
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
-                    tma_load_3d(sQ + kb * 16384, &tmQKV, &q_full, q_col + kb * 64, q_blk * 128, b);
+                    tma_load_3d(sQ + kb * 16384, &tmQKV, &q_full, q_col + kb * 64, p.q_lo + q_blk * 128, b);
                 for (int g = 0; g < 2 * nkb; ++g, ++gk) {
                     const int j = g % nkb, st = gk & 1;
                     if (!mbar_wait(&k_empty[st], ((gk >> 1) & 1) ^ 1, abortp)) { ok = false; break; }
@@ -295,8 +298,8 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
                 const int col = hf * (HD / 2) + ch * 32;
                 tmem_ld32(lane_base + O_COL + (it & 1) * 128 + col, v);
                 tmem_ld_wait();
-                if (q < L) {
-                    __nv_bfloat16* dst = p.out + ((size_t)b * L + q) * (size_t)(p.nq * HD) + h * HD + col;
+                if (q < p.q_cnt) {
+                    __nv_bfloat16* dst = p.out + ((size_t)b * p.q_cnt + q) * (size_t)(p.nq * HD) + h * HD + col;
 #pragma unroll
                     for (int g4 = 0; g4 < 4; ++g4) {
                         uint4 ov;

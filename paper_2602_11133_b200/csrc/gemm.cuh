@@ -42,10 +42,14 @@ struct GemmParams {
     int32_t* status;              // set non-zero when a bounded wait expired (nullable)
     int split_k;                  // EPI_PARTIAL: number of K ranges (>= 1); otherwise ignored
     float* partial;               // EPI_PARTIAL: [split_k][M][N] fp32
-    // EPI_QKV only: C = qkv [M, (nq + 2 nkv) * hd]; rows are (sequence, position) = (row / L, row % L)
+    // EPI_QKV only: C = qkv [B * L, (nq + 2 nkv) * hd].  The launch covers rows_per_seq consecutive canvas
+    // positions of every sequence, starting at pos0: input row r is (sequence, position) =
+    // (r / rows_per_seq, pos0 + r % rows_per_seq) and lands in row sequence * L + position of C and of V^T.
+    // The whole canvas is rows_per_seq = L, pos0 = 0; a block-wise KV cache recomputes one block's rows.
     __nv_bfloat16* vt;            // [B * nkv * hd, Lp] V transposed
     const float2* rope_cs;        // [max_seq, hd / 2] (cos, sin)
     int L, Lp, nq, nkv, hd;
+    int rows_per_seq, pos0;
     // EPI_STATS only
     const int32_t* d_R;           // number of active rows (device)
     const int32_t* rows;          // [R] flat canvas index b*L+i of each active row
@@ -56,8 +60,8 @@ struct GemmParams {
     // sampling-based finalisation (inv_temperature > 0): each row also draws a token from softmax(l / T)
     float inv_temperature;
     unsigned long long sample_seed;
-    const int32_t* d_step;        // device step counter (nullable: then step_value)
-    int step_value;
+    const int32_t* d_seq_steps;   // generate loop: steps_used of sequence b at d_seq_steps[4 * b] (nullable: then
+    int step_value;               // step_value); b = flat canvas index / L
     float2* partials2;            // [chunks][R_pad] (best perturbed score, bitcast token)
     int R_pad;                    // row capacity of one chunk of partials (multiple of 128)
 };
@@ -110,7 +114,8 @@ __device__ __forceinline__ void stats_row_init(const GemmParams& p, int row, Sta
         st.bump_v = p.bump_val[flat];
     }
     if (p.inv_temperature > 0.f) {
-        const unsigned long long step = (unsigned long long)(p.d_step ? *p.d_step : p.step_value);
+        const unsigned long long step =
+            (unsigned long long)(p.d_seq_steps ? p.d_seq_steps[4 * (flat / p.L)] : p.step_value);
         st.key = mix64(p.sample_seed ^ (step << 40) ^ (unsigned long long)flat);
     }
 }
@@ -159,7 +164,8 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
         }
     } else if (EPI == EPI_QKV) {
         const int hd = p.hd, half = hd >> 1;
-        const int seq = row / p.L, pos = row - seq * p.L;
+        const int seq = row / p.rows_per_seq, pos = p.pos0 + (row - seq * p.rows_per_seq);
+        const size_t dst_row = (size_t)seq * p.L + pos;
 #pragma unroll 1
         for (int hh = 0; hh < BN / hd; ++hh) {
             const int col_base = n_blk * BN + hh * hd;
@@ -175,7 +181,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
                     tmem_ld_wait();
                     if (row < p.M) {
                         const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cs + (size_t)pos * half + q * 32);
-                        __nv_bfloat16* dlo = p.C + (size_t)row * p.ldc + col_base + q * 32;
+                        __nv_bfloat16* dlo = p.C + dst_row * p.ldc + col_base + q * 32;
                         __nv_bfloat16* dhi = dlo + half;
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {

@@ -34,17 +34,21 @@ __device__ __forceinline__ float block_sum(float v, float* scratch /* >= 33 floa
 }
 
 // h[row, :] = E[token of that row, :]     one CTA per row, 16-byte copies (d multiple of 8).
-// With seq_map the rows are those of a compacted batch: row = (b', i) reads tokens[seq_map[b'], i].
+// The launch covers rows_per_seq consecutive canvas positions of every sequence, starting at pos0 (the whole
+// canvas: L, 0): row r is (slot, position) = (r / rows_per_seq, pos0 + r % rows_per_seq).
+// With seq_map the slots are those of a compacted batch: slot b' reads tokens[seq_map[b'], position].
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E,
-                             __nv_bfloat16* __restrict__ h, int d, int L, const int32_t* __restrict__ seq_map) {
+                             __nv_bfloat16* __restrict__ h, int d, int L, const int32_t* __restrict__ seq_map,
+                             int rows_per_seq, int pos0) {
     grid_launch_dependents();
     grid_dependency_wait();
     const int row = blockIdx.x;
-    int src_row = row;
+    int b = row / rows_per_seq;
     if (seq_map) {
-        const int b = seq_map[row / L];                 // unused slots (-1) compute on sequence 0; nobody reads them
-        src_row = (b < 0 ? 0 : b) * L + row % L;
+        b = seq_map[b];                                 // unused slots (-1) compute on sequence 0; nobody reads them
+        b = b < 0 ? 0 : b;
     }
+    const int src_row = b * L + pos0 + row % rows_per_seq;
     const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[src_row] * d);
     uint4* dst = reinterpret_cast<uint4*>(h + (size_t)row * d);
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = src[i];
@@ -187,14 +191,15 @@ __global__ void __launch_bounds__(512) splitk_reduce_norm_kernel(const float* __
 // Active rows of the step: every position of [lo_b, hi_b) that holds mask_id, in (b, i) order.
 // Single CTA.  rows_out[r] = b*L + i (index into the caller's [B, L] arrays); rows[r] = the same row's index
 // in the forward pass's activation matrix, which differs when finished sequences were compacted away
-// (seq_map: compact slot -> sequence; n_seq slots).  *d_R = count.  With `state`, each sequence uses its
+// (seq_map: compact slot -> sequence; n_seq slots) or when the pass covered only positions pos0 ..
+// pos0 + rows_per_seq - 1 of every sequence (the whole canvas: rows_per_seq = L, pos0 = 0).  *d_R = count.  With `state`, each sequence uses its
 // own block and finished sequences contribute nothing.
 __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restrict__ tokens, int B, int L,
                                                           int32_t mask_id, int blk_lo, int blk_hi,
                                                           const SeqState* __restrict__ state, int P, int block_len,
                                                           int n_blocks, const int32_t* __restrict__ seq_map,
                                                           int32_t* __restrict__ rows, int32_t* __restrict__ rows_out,
-                                                          int32_t* __restrict__ d_R) {
+                                                          int32_t* __restrict__ d_R, int rows_per_seq, int pos0) {
     grid_launch_dependents();
     grid_dependency_wait();
     __shared__ int warp_counts[32];
@@ -222,7 +227,7 @@ __global__ void __launch_bounds__(1024) build_rows_kernel(const int32_t* __restr
             for (int w = 0; w < wid; ++w) off += warp_counts[w];
             if (c) {
                 const int r = off + __popc(bal & ((1u << ln) - 1u));
-                rows[r] = slot * L + i;
+                rows[r] = slot * rows_per_seq + (i - pos0);
                 rows_out[r] = b * L + i;
             }
             __syncthreads();

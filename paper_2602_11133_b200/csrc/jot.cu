@@ -5,8 +5,10 @@
 #include <cudaTypedefs.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstddef>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -294,7 +296,18 @@ struct jot_model {
     AcceptParamsDev* params_dev;
     // activation tensor maps, re-encoded when (B, L) changes
     int map_B = -1, map_L = -1;
-    CUtensorMap tm_a, tm_attn, tm_act, tm_hsel, tm_qkv3, tm_vt;
+    CUtensorMap tm_hsel, tm_qkv3, tm_vt;
+    // A-operand maps of the projections for a pass over M rows (rows past M read as zero without memory
+    // traffic): one set for the whole canvas, one for the rows of a block
+    struct ActMaps { int M = -1; CUtensorMap a, attn, act; };
+    ActMaps maps_full, maps_span;
+    // block-wise KV cache (caller's memory, optional): per layer the rotated Q/K rows and V^T of the whole canvas
+    uint8_t* kv_base = nullptr;
+    size_t kv_bytes = 0;
+    std::vector<__nv_bfloat16*> kv_qkv, kv_vt;
+    std::vector<CUtensorMap> kv_tm_qkv3, kv_tm_vt;
+    int kv_map_B = -1, kv_map_L = -1;       // geometry the per-layer maps were encoded for
+    int kv_valid_B = -1, kv_valid_L = -1;   // geometry of the last refresh (block passes need one)
     int32_t* h_pinned = nullptr;    // pinned host words for loop control read-back (two 4-word slots, then SeqState)
     cudaEvent_t step_done[2] = {nullptr, nullptr};
     // optional per-kernel-class timing with CUDA events on the launching stream
@@ -399,9 +412,7 @@ int encode_activation_maps(jot_model* m, int B, int L) {
     const int M = B * L;
     const int qkv_cols = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
     const int Lp = (int)align_up((size_t)L, 8);
-    JOT_TRY(make_map_2d(m->di, &m->tm_a, m->a, M, c.d_model, c.d_model, 128));
-    JOT_TRY(make_map_2d(m->di, &m->tm_attn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim, 128));
-    JOT_TRY(make_map_2d(m->di, &m->tm_act, m->act, M, c.d_ff, c.d_ff, 128));
+    (void)M;
     JOT_TRY(make_map_2d(m->di, &m->tm_hsel, m->hsel, m->R_cap, c.d_model, c.d_model, 128));
     JOT_TRY(make_map_qkv(m->di, &m->tm_qkv3, m->qkv, B, L, qkv_cols));
     JOT_TRY(make_map_2d(m->di, &m->tm_vt, m->vt, (uint64_t)B * c.n_kv_heads * c.head_dim, L, Lp, c.head_dim));
@@ -410,19 +421,67 @@ int encode_activation_maps(jot_model* m, int B, int L) {
     return JOT_OK;
 }
 
-// Transformer body: tokens [B, L] -> residual stream m->h [B*L, d] (before the final norm).
-// B sequences are processed; with seq_map they are the compacted batch (slot -> sequence of d_tokens).
-int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream_t st, const int32_t* seq_map = nullptr) {
+int encode_act_maps(jot_model* m, jot_model::ActMaps* am, int M) {
+    if (am->M == M) return JOT_OK;
     const jot_model_config& c = m->cfg;
-    const int M = B * L, d = c.d_model, hd = c.head_dim, nq = c.n_q_heads, nkv = c.n_kv_heads;
+    JOT_TRY(make_map_2d(m->di, &am->a, m->a, M, c.d_model, c.d_model, 128));
+    JOT_TRY(make_map_2d(m->di, &am->attn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim, 128));
+    JOT_TRY(make_map_2d(m->di, &am->act, m->act, M, c.d_ff, c.d_ff, 128));
+    am->M = M;
+    return JOT_OK;
+}
+
+// Per-layer slices of an attached KV cache for canvases of B x L, and their tensor maps.
+size_t kv_layer_bytes(const jot_model_config* c, int max_batch, int max_seq, size_t* vt_off) {
+    const size_t qkv_cols = (size_t)(c->n_q_heads + 2 * c->n_kv_heads) * c->head_dim;
+    const size_t q = align_up((size_t)max_batch * max_seq * qkv_cols * 2, 1024);
+    const size_t v = align_up((size_t)max_batch * c->n_kv_heads * c->head_dim * align_up((size_t)max_seq, 8) * 2, 1024);
+    if (vt_off) *vt_off = q;
+    return q + v;
+}
+
+int encode_kv_maps(jot_model* m, int B, int L) {
+    if (m->kv_map_B == B && m->kv_map_L == L) return JOT_OK;
+    const jot_model_config& c = m->cfg;
+    const int qkv_cols = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+    const int Lp = (int)align_up((size_t)L, 8);
+    for (int l = 0; l < c.n_layers; ++l) {
+        JOT_TRY(make_map_qkv(m->di, &m->kv_tm_qkv3[l], m->kv_qkv[l], B, L, qkv_cols));
+        JOT_TRY(make_map_2d(m->di, &m->kv_tm_vt[l], m->kv_vt[l], (uint64_t)B * c.n_kv_heads * c.head_dim, L, Lp, c.head_dim));
+    }
+    m->kv_map_B = B;
+    m->kv_map_L = L;
+    m->kv_valid_B = m->kv_valid_L = -1;      // another geometry lays the rows out differently
+    return JOT_OK;
+}
+
+// Which rows a pass covers: positions pos0 .. pos0 + Lr - 1 of every sequence; use_cache: the rotated Q/K
+// rows and V^T of every layer live in the attached KV cache instead of the one scratch buffer, so that a
+// later pass over one block finds the rest of the canvas there.
+struct FwdSpan {
+    int Lr, pos0;
+    bool use_cache;
+};
+
+// Transformer body: tokens [B, L] -> residual stream m->h [B*Lr, d] (before the final norm).
+// B sequences are processed; with seq_map they are the compacted batch (slot -> sequence of d_tokens).
+int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream_t st, const int32_t* seq_map = nullptr,
+                 const FwdSpan* span = nullptr) {
+    const jot_model_config& c = m->cfg;
+    const int Lr = span ? span->Lr : L, pos0 = span ? span->pos0 : 0;
+    const bool cached = span && span->use_cache;
+    const int M = B * Lr, d = c.d_model, hd = c.head_dim, nq = c.n_q_heads, nkv = c.n_kv_heads;
     const int qkv_cols = (nq + 2 * nkv) * hd;
     const int Lp = (int)align_up((size_t)L, 8);
     JOT_TRY(encode_activation_maps(m, B, L));
+    jot_model::ActMaps& am = (Lr == L) ? m->maps_full : m->maps_span;
+    JOT_TRY(encode_act_maps(m, &am, M));
+    if (cached) JOT_TRY(encode_kv_maps(m, B, L));
     int32_t* status = m->ctrl;
 
     {
         ProfScope ps(m, JOT_PROF_EMBED, st);
-        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d, L, seq_map);
+        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d, L, seq_map, Lr, pos0);
     }
     JOT_TRY(launch_check());
     bool norm_ready = false;          // true when a fused split-K tail has already written the next norm into m->a
@@ -433,28 +492,32 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
             JOT_TRY(launch_check());
         }
         GemmParams p{};
-        p.M = M; p.N = qkv_cols; p.K = d; p.C = m->qkv; p.ldc = qkv_cols; p.status = status;
+        p.M = M; p.N = qkv_cols; p.K = d; p.C = cached ? m->kv_qkv[l] : m->qkv; p.ldc = qkv_cols; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_QKV, st);
-            p.vt = m->vt; p.rope_cs = m->rope_cs; p.L = L; p.Lp = Lp; p.nq = nq; p.nkv = nkv; p.hd = hd;
-            JOT_TRY(run_gemm(m->di, m->tm_a, m->wqkv[l], EPI_QKV, p, st));
+            p.vt = cached ? m->kv_vt[l] : m->vt; p.rope_cs = m->rope_cs; p.L = L; p.Lp = Lp; p.nq = nq; p.nkv = nkv;
+            p.hd = hd; p.rows_per_seq = Lr; p.pos0 = pos0;
+            JOT_TRY(run_gemm(m->di, am.a, m->wqkv[l], EPI_QKV, p, st));
         }
         AttnParams ap{};
         ap.B = B; ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
+        ap.q_lo = pos0; ap.q_cnt = Lr;
         ap.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
-        const long items = (long)B * nq * ((L + 127) / 128);
+        const long items = (long)B * nq * ((Lr + 127) / 128);
         dim3 grid((unsigned)(items < m->di->sms ? items : m->di->sms));
         {
             ProfScope ps(m, JOT_PROF_ATTENTION, st);
-            if (hd == 128) JOT_TRY(launch_attention_t<128>(ap, m->tm_qkv3, m->tm_vt, grid, st));
-            else JOT_TRY(launch_attention_t<64>(ap, m->tm_qkv3, m->tm_vt, grid, st));
+            const CUtensorMap& tq = cached ? m->kv_tm_qkv3[l] : m->tm_qkv3;
+            const CUtensorMap& tv = cached ? m->kv_tm_vt[l] : m->tm_vt;
+            if (hd == 128) JOT_TRY(launch_attention_t<128>(ap, tq, tv, grid, st));
+            else JOT_TRY(launch_attention_t<64>(ap, tq, tv, grid, st));
         }
         p = GemmParams{};
         p.M = M; p.N = d; p.K = nq * hd; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_O, st);
             NormAfter na{m->mlp_norm[l], m->a, c.rms_eps, false};
-            JOT_TRY(run_gemm(m->di, m->tm_attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes, &na));
+            JOT_TRY(run_gemm(m->di, am.attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes, &na));
             norm_ready = na.done;
         }
         if (!norm_ready) {
@@ -466,14 +529,14 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = 2 * c.d_ff; p.K = d; p.C = m->act; p.ldc = c.d_ff; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_GATE_UP, st);
-            JOT_TRY(run_gemm(m->di, m->tm_a, m->wgu[l], EPI_SWIGLU, p, st));
+            JOT_TRY(run_gemm(m->di, am.a, m->wgu[l], EPI_SWIGLU, p, st));
         }
         p = GemmParams{};
         p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_DOWN, st);
             NormAfter na{l + 1 < c.n_layers ? m->attn_norm[l + 1] : nullptr, m->a, c.rms_eps, false};
-            JOT_TRY(run_gemm(m->di, m->tm_act, m->wdown[l], EPI_STORE, p, st, m->splitk, kSplitKBytes,
+            JOT_TRY(run_gemm(m->di, am.act, m->wdown[l], EPI_STORE, p, st, m->splitk, kSplitKBytes,
                              na.gain ? &na : nullptr));
             norm_ready = na.done;
         }
@@ -482,12 +545,14 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
 }
 
 // hsel (active rows, already gathered) -> merged statistics scattered to the [B, L] outputs
-// Sampling-based finalisation of the head: temperature > 0 turns it on; the step index comes from the
-// device counter when d_step is given (generate loop), else from step_value.
+// Sampling-based finalisation of the head: temperature > 0 turns it on; the step index of a row is its
+// sequence's own count of denoising steps so far when d_seq_steps is given (generate loop: the draw then does
+// not depend on what else is in the batch), else step_value.
 struct HeadSampling {
     float temperature = 0.f;
     unsigned long long seed = 0;
-    const int32_t* d_step = nullptr;
+    const int32_t* d_seq_steps = nullptr;
+    int L = 1;
     int step_value = 0;
     int32_t* sampled = nullptr;      // [B, L] output
 };
@@ -496,6 +561,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
                       float* top2, float* sumexp, int32_t* argmax, int M, cudaStream_t st,
                       const HeadSampling* hs = nullptr) {
     const jot_model_config& c = m->cfg;
+    if (M <= 0) return JOT_OK;                       // an empty block range has no active rows
     GemmParams p{};
     p.M = m->R_cap; p.N = c.vocab; p.K = c.d_model; p.status = m->ctrl;
     p.d_R = m->ctrl + 1; p.rows = m->rows_out; p.bump_id = bump_id; p.bump_val = bump_val;
@@ -503,8 +569,8 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     p.partials = m->partials; p.R_pad = m->R_cap;
     const bool sampling = hs && hs->temperature > 0.f;
     if (sampling) {
-        p.inv_temperature = 1.f / hs->temperature; p.sample_seed = hs->seed; p.d_step = hs->d_step;
-        p.step_value = hs->step_value; p.partials2 = m->partials2;
+        p.inv_temperature = 1.f / hs->temperature; p.sample_seed = hs->seed; p.d_seq_steps = hs->d_seq_steps;
+        p.L = hs->L; p.step_value = hs->step_value; p.partials2 = m->partials2;
     }
     // few active rows: the head streams W once and is bandwidth bound -> narrow tiles balance the SMs best;
     // many rows: CTA pairs (256 x 256 tiles) halve the W bytes each SM takes in
@@ -747,7 +813,7 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
     {
         ProfScope ps(m, JOT_PROF_ROWS, st);
         launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, nullptr, m->rows, m->rows_out,
-                                              m->ctrl + 1);
+                                              m->ctrl + 1, L, 0);
         JOT_TRY(launch_check());
         launch_k(gather_rows_kernel, dim3(B * L), dim3(128), 0, st, (const __nv_bfloat16*)d_hidden, m->hsel, m->cfg.d_model, m->rows,
                                                   m->ctrl + 1);
@@ -758,26 +824,78 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
     return read_status(m, st);
 }
 
-int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi, int exclude_mask_token,
-                     const int32_t* d_bump_id, const float* d_bump_val, float* d_top1, float* d_top2, float* d_sumexp,
-                     int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled, void* stream) {
+namespace {
+int denoise_step_impl(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi, int exclude_mask_token,
+                      const int32_t* d_bump_id, const float* d_bump_val, float* d_top1, float* d_top2, float* d_sumexp,
+                      int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled, void* stream,
+                      const FwdSpan* span) {
     JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
     HeadSampling hs;
     JOT_TRY(head_sampling_from(sampling, d_sampled, &hs));
     cudaStream_t st = (cudaStream_t)stream;
-    JOT_TRY(forward_body(m, d_tokens, B, L, st));
+    const int Lr = span ? span->Lr : L, pos0 = span ? span->pos0 : 0;
+    JOT_TRY(forward_body(m, d_tokens, B, L, st, nullptr, span));
     {
         ProfScope ps(m, JOT_PROF_ROWS, st);
         launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, d_tokens, B, L, m->cfg.mask_id, blk_lo, blk_hi, nullptr, 0, 0, 0, nullptr, m->rows, m->rows_out,
-                                              m->ctrl + 1);
+                                              m->ctrl + 1, Lr, pos0);
         JOT_TRY(launch_check());
-        launch_k(rmsnorm_kernel, dim3(B * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
+        launch_k(rmsnorm_kernel, dim3(std::max(1, B * (blk_hi - blk_lo))), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model, m->cfg.rms_eps, m->rows,
                                               m->ctrl + 1);
         JOT_TRY(launch_check());
     }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
                               B * (blk_hi - blk_lo), st, &hs));
     return read_status(m, st);
+}
+}  // namespace
+
+int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi, int exclude_mask_token,
+                     const int32_t* d_bump_id, const float* d_bump_val, float* d_top1, float* d_top2, float* d_sumexp,
+                     int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled, void* stream) {
+    return denoise_step_impl(m, d_tokens, B, L, blk_lo, blk_hi, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2,
+                             d_sumexp, d_argmax, sampling, d_sampled, stream, nullptr);
+}
+
+size_t jot_kv_cache_bytes(const jot_model_config* cfg, int max_batch, int max_seq) {
+    if (!config_ok(cfg) || max_batch <= 0 || max_seq <= 0) return 0;
+    return (size_t)cfg->n_layers * kv_layer_bytes(cfg, max_batch, max_seq, nullptr) + 1024;
+}
+
+int jot_attach_kv_cache(jot_model* m, void* d_cache, size_t bytes) {
+    if (!m) return JOT_ERR_ARG;
+    m->kv_map_B = m->kv_map_L = m->kv_valid_B = m->kv_valid_L = -1;
+    m->kv_base = nullptr;
+    m->kv_bytes = 0;
+    if (!d_cache) return JOT_OK;                                   // detach
+    if (reinterpret_cast<uintptr_t>(d_cache) & 1023) return JOT_ERR_ARG;
+    if (bytes < jot_kv_cache_bytes(&m->cfg, m->max_batch, m->max_seq)) return JOT_ERR_WORKSPACE;
+    size_t vt_off = 0;
+    const size_t per_layer = kv_layer_bytes(&m->cfg, m->max_batch, m->max_seq, &vt_off);
+    const int n = m->cfg.n_layers;
+    m->kv_qkv.resize(n); m->kv_vt.resize(n); m->kv_tm_qkv3.resize(n); m->kv_tm_vt.resize(n);
+    for (int l = 0; l < n; ++l) {
+        uint8_t* base = (uint8_t*)d_cache + (size_t)l * per_layer;
+        m->kv_qkv[l] = (__nv_bfloat16*)base;
+        m->kv_vt[l] = (__nv_bfloat16*)(base + vt_off);
+    }
+    m->kv_base = (uint8_t*)d_cache;
+    m->kv_bytes = bytes;
+    return JOT_OK;
+}
+
+int jot_denoise_step_cached(jot_model* m, const int32_t* d_tokens, int B, int L, int blk_lo, int blk_hi, int refresh,
+                            int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val, float* d_top1,
+                            float* d_top2, float* d_sumexp, int32_t* d_argmax, const jot_sampling* sampling,
+                            int32_t* d_sampled, void* stream) {
+    if (!m || !m->kv_base) return JOT_ERR_ARG;
+    if (blk_lo >= blk_hi) return JOT_ERR_ARG;
+    if (!refresh && (m->kv_valid_B != B || m->kv_valid_L != L)) return JOT_ERR_ARG;     // nothing cached for this canvas
+    const FwdSpan span = refresh ? FwdSpan{L, 0, true} : FwdSpan{blk_hi - blk_lo, blk_lo, true};
+    const int rc = denoise_step_impl(m, d_tokens, B, L, blk_lo, blk_hi, exclude_mask_token, d_bump_id, d_bump_val, d_top1,
+                                     d_top2, d_sumexp, d_argmax, sampling, d_sampled, stream, &span);
+    if (rc == JOT_OK && refresh) { m->kv_valid_B = B; m->kv_valid_L = L; }
+    return rc;
 }
 
 int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask_id, int32_t* d_tokens, int B, int L,
@@ -820,6 +938,7 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         if (!params_ok(params + i)) return JOT_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     static_assert(sizeof(AcceptParamsDev) == sizeof(jot_params), "parameter struct layouts must agree");
+    static_assert(sizeof(SeqState) == 16 && offsetof(SeqState, steps_used) == 8, "the head reads steps_used at int 2 of 4");
     JOT_CUDA(cudaMemcpyAsync(m->params_dev, params, (size_t)n_par * sizeof(jot_params), cudaMemcpyHostToDevice, st));
     launch_k(init_canvas_kernel, dim3((B * L + 255) / 256), dim3(256), 0, st, d_prompt, m->canvas, B, P, gen->gen_len, m->cfg.mask_id,
                                                            m->state);
@@ -845,17 +964,74 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         if (!*finished) B_act = w[2];
         return JOT_OK;
     };
-    // sampling-based finalisation: the step index lives on the device (advanced by the acceptance kernel), so a
+    // sampling-based finalisation: the step index is read from the per-sequence state on the device, so a
     // captured step can be replayed unchanged
     const bool sampling = gen->temperature > 0.f;
     HeadSampling hs;
     if (sampling) {
         hs.temperature = gen->temperature;
         hs.seed = ((unsigned long long)gen->seed_hi << 32) | gen->seed_lo;
-        hs.d_step = m->ctrl + 4;
+        hs.d_seq_steps = reinterpret_cast<const int32_t*>(m->state) + 2;      // SeqState::steps_used
+        hs.L = L;
         hs.sampled = m->g_sampled;
     }
-    JOT_CUDA(cudaMemsetAsync(m->ctrl + 4, 0, 4, st));
+    if (gen->kv_cache) {
+        // Block-wise KV cache: every sequence works on the same block.  The first step of a block runs the whole
+        // canvas and leaves every layer's keys and values in the cache; the block's other steps run only the
+        // block's rows against it.  The host reads the block's outcome after every step (what runs next depends
+        // on it), so this loop is not pipelined.
+        if (!m->kv_base) return JOT_ERR_ARG;
+        const int Lb = gen->block_len;
+        int n_passes = 0;
+        for (int blk = 0; blk < nb; ++blk) {
+            const int lo = P + blk * Lb, hi = lo + Lb;
+            for (int s = 0; s < Tb; ++s) {
+                JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
+                const FwdSpan span = (s == 0) ? FwdSpan{L, 0, true} : FwdSpan{Lb, lo, true};
+                JOT_TRY(forward_body(m, m->canvas, B, L, st, nullptr, &span));
+                {
+                    ProfScope ps(m, JOT_PROF_ROWS, st);
+                    launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, m->canvas, B, L, m->cfg.mask_id, lo, hi, nullptr, 0,
+                             0, 0, nullptr, m->rows, m->rows_out, m->ctrl + 1, span.Lr, span.pos0);
+                    JOT_TRY(launch_check());
+                    launch_k(rmsnorm_kernel, dim3(B * Lb), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model,
+                             m->cfg.rms_eps, m->rows, m->ctrl + 1);
+                    JOT_TRY(launch_check());
+                }
+                JOT_TRY(lm_head_from_hsel(m, gen->exclude_mask_token, d_bump_id, d_bump_val, m->g_top1, m->g_top2,
+                                          m->g_sumexp, m->g_argmax, B * Lb, st, &hs));
+                AcceptArgs a{};
+                a.params = m->params_dev; a.per_seq_params = per_seq_params ? 1 : 0;
+                a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
+                a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp;
+                a.argmax = sampling ? m->g_sampled : m->g_argmax;
+                a.state = m->state; a.lockstep = 1; a.blk_lo = lo; a.blk_hi = hi;
+                a.k_transfer = Lb / Tb + (s < Lb % Tb ? 1 : 0);
+                a.n_unfinished = m->ctrl + 2;
+                if (trace) {
+                    a.exit_step = trace->d_exit_step; a.exit_reason = trace->d_exit_reason;
+                    a.mean_ratio = trace->d_mean_ratio; a.n_candidates = trace->d_n_candidates;
+                }
+                {
+                    ProfScope ps(m, JOT_PROF_ACCEPT, st);
+                    JOT_TRY(launch_accept(a, st));
+                }
+                JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 16, cudaMemcpyDeviceToHost, st));
+                JOT_CUDA(cudaStreamSynchronize(st));
+                if (m->h_pinned[0]) return JOT_ERR_TIMEOUT;
+                ++n_passes;
+                if (m->h_pinned[2] == 0) break;              // no sequence has a masked position left in this block
+            }
+        }
+        m->kv_valid_B = m->kv_valid_L = -1;                  // the cache belongs to a canvas that is finished
+        JOT_CUDA(cudaMemcpyAsync(d_out_tokens, m->canvas, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
+        SeqState* hstate = reinterpret_cast<SeqState*>(m->h_pinned + 16);
+        JOT_CUDA(cudaMemcpyAsync(hstate, m->state, (size_t)B * sizeof(SeqState), cudaMemcpyDeviceToHost, st));
+        JOT_CUDA(cudaStreamSynchronize(st));
+        for (int b = 0; b < B; ++b) h_steps_used[b] = hstate[b].steps_used;
+        if (h_forward_passes) *h_forward_passes = n_passes;
+        return JOT_OK;
+    }
     // everything one step enqueues, ending with the copy of the control words to the pinned slot it & 1
     auto enqueue_step = [&](int it, int Bf, const int32_t* seq_map) -> int {
         JOT_CUDA(cudaMemsetAsync(m->ctrl + 2, 0, 4, st));
@@ -868,7 +1044,7 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         {
             ProfScope ps(m, JOT_PROF_ROWS, st);
             launch_k(build_rows_kernel, dim3(1), dim3(1024), 0, st, m->canvas, Bf, L, m->cfg.mask_id, 0, 0, m->state, P,
-                     gen->block_len, nb, seq_map, m->rows, m->rows_out, m->ctrl + 1);
+                     gen->block_len, nb, seq_map, m->rows, m->rows_out, m->ctrl + 1, L, 0);
             JOT_TRY(launch_check());
             launch_k(rmsnorm_kernel, dim3(Bf * L), dim3(256), 0, st, m->h, m->final_norm, m->hsel, m->cfg.d_model,
                      m->cfg.rms_eps, m->rows, m->ctrl + 1);
@@ -881,7 +1057,6 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
         a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
         a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp;
         a.argmax = sampling ? m->g_sampled : m->g_argmax;       // the token a finalised position receives
-        a.step_counter = m->ctrl + 4;
         a.step_index = it + 1;                       // only reaches the optional exit-step output, unused here
         a.state = m->state; a.P = P; a.block_len = gen->block_len; a.n_blocks = nb; a.steps_per_block = Tb;
         a.n_unfinished = m->ctrl + 2;

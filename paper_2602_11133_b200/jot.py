@@ -20,7 +20,7 @@ EXPORTS = [
     "jot_status_string", "jot_last_cuda_error", "jot_workspace_bytes", "jot_init_model", "jot_free_model",
     "jot_denoise_step", "jot_lm_head_stats", "jot_accept_freeze", "jot_generate", "jot_gemm_bf16",
     "jot_launch_count", "jot_profile", "jot_profile_read", "jot_gemm_bf16_noalloc",
-    "jot_selftest_wait_expiry",
+    "jot_selftest_wait_expiry", "jot_kv_cache_bytes", "jot_attach_kv_cache", "jot_denoise_step_cached",
 ]
 
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -72,7 +72,7 @@ class Sampling(C.Structure):
 class GenConfig(C.Structure):
     _fields_ = [("gen_len", C.c_int32), ("steps", C.c_int32), ("block_len", C.c_int32),
                 ("exclude_mask_token", C.c_int32), ("compact_finished", C.c_int32), ("use_cuda_graph", C.c_int32),
-                ("temperature", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
+                ("temperature", C.c_float), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32), ("kv_cache", C.c_int32)]
 
 
 class _Trace(C.Structure):
@@ -111,6 +111,12 @@ def _lib():
                      C.c_void_p, C.c_void_p, C.POINTER(Sampling), C.c_void_p, C.c_void_p]
         lib.jot_denoise_step.argtypes = [C.c_void_p, C.c_void_p] + step_args
         lib.jot_lm_head_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + step_args
+        lib.jot_kv_cache_bytes.restype = C.c_size_t
+        lib.jot_kv_cache_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int, C.c_int]
+        lib.jot_attach_kv_cache.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
+        lib.jot_denoise_step_cached.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                C.c_void_p, C.POINTER(Sampling), C.c_void_p, C.c_void_p]
         lib.jot_accept_freeze.argtypes = [C.POINTER(Params), C.c_int, C.c_int32, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                           C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
@@ -203,11 +209,43 @@ class Model:
         _check(lib.jot_init_model(C.byref(self.cfg), C.byref(w), max_batch, max_seq, base, nbytes, C.byref(handle)),
                "jot_init_model")
         self.handle = handle
+        self.kv_cache = None
 
     def close(self):
         if getattr(self, "handle", None):
             _lib().jot_free_model(self.handle)
             self.handle = None
+        self.kv_cache = None
+
+    # ---- block-wise KV cache -----------------------------------------------------------------------
+    def attach_kv_cache(self) -> int:
+        """Allocate the cache for (max_batch, max_seq) and hand it to the library; returns its size in bytes."""
+        nbytes = _lib().jot_kv_cache_bytes(C.byref(self.cfg), self.max_batch, self.max_seq)
+        if nbytes == 0:
+            raise JotError(-2, "jot_kv_cache_bytes")
+        self.kv_cache = torch.empty(nbytes + 1024, dtype=torch.uint8, device=self.workspace.device)
+        base = (self.kv_cache.data_ptr() + 1023) // 1024 * 1024
+        _check(_lib().jot_attach_kv_cache(self.handle, base, nbytes), "jot_attach_kv_cache")
+        return int(nbytes)
+
+    def detach_kv_cache(self) -> None:
+        _check(_lib().jot_attach_kv_cache(self.handle, None, 0), "jot_attach_kv_cache")
+        self.kv_cache = None
+
+    def denoise_step_cached(self, tokens: torch.Tensor, blk_lo: int, blk_hi: int, refresh: bool,
+                            out: Optional["Stats"] = None, exclude_mask_token: bool = True,
+                            bump_id: Optional[torch.Tensor] = None, bump_val: Optional[torch.Tensor] = None,
+                            sampling: Optional[Sampling] = None) -> "Stats":
+        B, L = tokens.shape
+        out = out or Stats.empty(B, L, tokens.device)
+        sp, d_sampled = _sampling_args(sampling, out, B, L, tokens.device)
+        _check(_lib().jot_denoise_step_cached(self.handle, _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo, blk_hi,
+                                              int(refresh), int(exclude_mask_token), _ptr(bump_id, torch.int32, "bump_id"),
+                                              _ptr(bump_val, torch.float32, "bump_val"), out.top1.data_ptr(),
+                                              out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), sp,
+                                              d_sampled, _stream()),
+               "jot_denoise_step_cached")
+        return out
 
     def __del__(self):
         try:
@@ -263,7 +301,7 @@ class Model:
     def generate(self, prompt: torch.Tensor, gen_len: int, steps: int, params, block_len: Optional[int] = None,
                  exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
                  bump_val: Optional[torch.Tensor] = None, compact_finished: bool = True, use_cuda_graph: bool = False,
-                 temperature: float = 0.0, seed: int = 0, trace: bool = False):
+                 temperature: float = 0.0, seed: int = 0, trace: bool = False, kv_cache: bool = False):
         """Returns (tokens [B, P+gen_len] int32 on device, steps_used list[int], forward_passes int), and a
         Trace as a fourth element when trace is set."""
         B, P = prompt.shape
@@ -275,7 +313,8 @@ class Model:
         else:
             parr = (Params * 1)(params)
         gen = GenConfig(gen_len, steps, block_len or gen_len, int(exclude_mask_token), int(compact_finished),
-                        int(use_cuda_graph), float(temperature), seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+                        int(use_cuda_graph), float(temperature), seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF,
+                        int(kv_cache))
         out = torch.empty(B, P + gen_len, dtype=torch.int32, device=prompt.device)
         used = (C.c_int32 * B)()
         passes = C.c_int32(0)
