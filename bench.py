@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # profiles/, keyed by kernel class and workload; removed (-> null) whenever the kernel changes afterwards.
 NCU_TRAFFIC = {
     ("llada8b", "gemm_gate_up"): 215.4e6,     # profiles/gemm_llada8b_m384.md
-    ("lmhead", "lm_head"): 1078.2e6,          # profiles/lm_head_pair_lmhead.md
+    ("lmhead", "lm_head"): 1067.0e6,          # profiles/lm_head_pair_lmhead.md
 }
 
 WORKLOADS = {
