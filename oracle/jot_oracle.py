@@ -24,7 +24,9 @@ choice is visible at the call site):
     details"); `schedule_after_exit=True` gives the other reading of
     Algorithm 1 (schedule ranks only what early exit left masked);
   * in block mode candidates are restricted to the current block while the
-    spatial window still sees the whole canvas.
+    spatial window still sees the whole canvas;
+  * the "global early-commit rule" of the related work is read as: mean top-2
+    logit gap of the candidates >= one threshold (see JotParams).
 
 Parity unpinned: the choice among those readings (no printed output of the
 paper distinguishes them).
@@ -44,7 +46,12 @@ class JotParams:
 
     gate = "ratio" is the paper's test r >= tau (Eq. 8).  gate = "maxprob" is the fixed probability gate the
     paper contrasts it with (Section 2: a position is finalised when its max probability clears a threshold,
-    0.9 in the compared system): p1 >= prob_threshold, no spatial modulation."""
+    0.9 in the compared system): p1 >= prob_threshold, no spatial modulation.  gate = "globalgap" is the
+    global early-commit rule the paper contrasts it with (Section 2: "once the top-2 confidence gap exceeds a
+    threshold, all remaining masked positions are finalized simultaneously"): the mean over the candidates of
+    the top-2 logit gap m1 - m2 is tested against gap_threshold and either every candidate exits or none does.
+    The compared system stages three thresholds over decoding progress (7.5 / 5.0 / 2.5, Section 5.1); here
+    the threshold is one input that a caller may change from step to step."""
     tau_max: float = 90.0
     tau_min: float = 1.0
     gamma: float = 0.5
@@ -52,6 +59,7 @@ class JotParams:
     eps: float = 1e-12
     gate: str = "ratio"
     prob_threshold: float = 0.9
+    gap_threshold: float = 5.0
 
 
 DREAM_DEFAULT = JotParams(90.0, 1.0, 0.5, 8)   # Table 1 caption
@@ -230,11 +238,19 @@ def accept_freeze(x: List[int], stats: dict, p: JotParams, mask_id: int, blk_lo:
     A = [i for i in range(blk_lo, blk_hi) if x0[i] == mask_id]          # Algorithm 1: M_n (in block)
     ratio, tau, near = {}, {}, []
     E = []
+    if p.gate == "globalgap" and A:                                       # global early commit (Section 2)
+        mean_gap = sum(stats[i].m1 - stats[i].m2 for i in A) / len(A)
+        if abs(mean_gap - p.gap_threshold) <= 1e-3 * abs(p.gap_threshold):
+            near = list(A)
+        if np.float32(mean_gap) >= np.float32(p.gap_threshold):           # decided in float32
+            E = list(A)
     for i in A:
         st = stats[i]
         r = confidence_ratio(st.p1, st.p2, p.eps)                         # Eq. 4
         t = position_threshold(x0, i, mask_id, p)                         # Eq. 5-7
         ratio[i], tau[i] = r, t
+        if p.gate == "globalgap":
+            continue
         if p.gate == "maxprob":                                           # fixed probability gate (Section 2)
             if abs(st.p1 - p.prob_threshold) <= 1e-3 * p.prob_threshold:
                 near.append(i)

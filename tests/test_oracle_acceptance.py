@@ -339,3 +339,45 @@ def test_probability_gate():
     p = jo.JotParams(gate="maxprob", prob_threshold=0.9)
     rep = jo.accept_freeze(x, stats, p, M, 2, 5, 0)
     assert rep.exited == [2, 4] and x == [7, 7, 60, M, 62]      # inclusive; a large ratio alone does not pass
+
+
+def test_global_gap_gate_commits_everything_or_nothing():
+    """Section 2: the global early-commit rule finalises all remaining masked positions at once when the top-2
+    gap clears a threshold.  Read as the mean logit gap of the candidates; hand-computed cases."""
+    # gaps 6, 2, 4 -> mean 4.0
+    mk = lambda: {2: stats_from_gap(60, 6.0, p1=0.5), 3: stats_from_gap(61, 2.0, p1=0.9), 4: stats_from_gap(62, 4.0, p1=0.2)}
+    x = canvas("rrmmm")
+    rep = jo.accept_freeze(x, mk(), jo.JotParams(gate="globalgap", gap_threshold=4.0), M, 2, 5, 0)
+    assert rep.exited == [2, 3, 4] and x == [7, 7, 60, 61, 62]          # inclusive, and uncapped
+    x = canvas("rrmmm")
+    rep = jo.accept_freeze(x, mk(), jo.JotParams(gate="globalgap", gap_threshold=4.5), M, 2, 5, 1)
+    assert rep.exited == [] and rep.scheduled == [3] and x == [7, 7, M, 61, M]   # below: plain schedule step
+    # only the candidates of the current block count: position 4 (gap 1) lies outside it -> mean (6 + 2) / 2 = 4,
+    # where the mean over all three masked positions would be 3
+    x = canvas("rrmmm")
+    st3 = mk()
+    st3[4] = stats_from_gap(62, 1.0, p1=0.2)
+    rep = jo.accept_freeze(x, st3, jo.JotParams(gate="globalgap", gap_threshold=4.0), M, 2, 4, 0)
+    assert rep.exited == [2, 3] and x == [7, 7, 60, 61, M]
+    # a single very confident position does not commit the rest (the per-token ratio gate would exit it)
+    st = {2: stats_from_gap(60, 12.0), 3: stats_from_gap(61, 0.0), 4: stats_from_gap(62, 0.0)}
+    x = canvas("rrmmm")
+    assert jo.accept_freeze(x, st, jo.JotParams(gate="globalgap", gap_threshold=5.0), M, 2, 5, 0).exited == []
+    x = canvas("rrmmm")
+    assert jo.accept_freeze(x, st, jo.DREAM_DEFAULT, M, 2, 5, 0).exited == [2]
+    # near the threshold every candidate is reported
+    x = canvas("rrmmm")
+    rep = jo.accept_freeze(x, mk(), jo.JotParams(gate="globalgap", gap_threshold=4.0 * (1 + 5e-4)), M, 2, 5, 0)
+    assert rep.near_margin == [2, 3, 4]
+
+
+def test_global_gap_gate_in_the_loop():
+    """Threshold -inf-like: the first step commits the whole block (steps_used = number of blocks);
+    threshold +inf-like: plain schedule decoding, exactly T steps."""
+    prompt = [7] * 4
+    def stats_fn(x, rows):
+        return {i: stats_from_gap(100 + i, 3.0, p1=0.5 + 0.001 * i) for i in rows}
+    t = jo.generate(None, prompt, 8, 8, jo.JotParams(gate="globalgap", gap_threshold=-1e30), M, block_len=4, stats_fn=stats_fn)
+    assert t.steps_used == 2 and t.x[4:] == [104 + j for j in range(8)]
+    t = jo.generate(None, prompt, 8, 8, jo.JotParams(gate="globalgap", gap_threshold=1e30), M, block_len=4, stats_fn=stats_fn)
+    assert t.steps_used == 8 and all(len(r.exited) == 0 and len(r.scheduled) == 1 for r in t.reports)

@@ -12,7 +12,10 @@ import test_oracle_model as pins_m
 from oracle import jot_oracle as jo
 from oracle import model_oracle as mo
 
-ACCEPT_PINS = [getattr(pins_a, n) for n in dir(pins_a) if n.startswith("test_")]
+# the pins of the global early-commit gate are checked against their own planted mistakes below: the
+# rewritten decision rules of accept_variant() do not know that gate, so those pins would "notice" anything
+ACCEPT_PINS = [getattr(pins_a, n) for n in dir(pins_a) if n.startswith("test_") and not n.startswith("test_global_gap")]
+GAP_PINS = [getattr(pins_a, n) for n in dir(pins_a) if n.startswith("test_global_gap")]
 MODEL_PINS = [pins_m.test_rope_closed_form, pins_m.test_rmsnorm_closed_form,
               pins_m.test_attention_rows_average_values_and_see_everything,
               pins_m.test_forward_matches_independent_restatement, pins_m.test_bidirectional_not_causal,
@@ -163,6 +166,47 @@ DECISION_MUTATIONS = {
 def test_decision_pins_catch(name, monkeypatch):
     monkeypatch.setattr(jo, "accept_freeze", accept_variant(**DECISION_MUTATIONS[name]))
     assert some_pin_fails(ACCEPT_PINS), f"no pin noticed: {name}"
+
+
+def gap_variant(kind):
+    """accept_freeze whose global early-commit branch carries one planted mistake."""
+    orig = jo.accept_freeze
+
+    def fn(x, stats, p, mask_id, blk_lo, blk_hi, k_transfer, schedule_after_exit=False, tokens=None):
+        if p.gate != "globalgap":
+            return orig(x, stats, p, mask_id, blk_lo, blk_hi, k_transfer, schedule_after_exit, tokens)
+        A = [i for i in range(blk_lo, blk_hi) if x[i] == mask_id]
+        pool = [i for i in range(len(x)) if x[i] == mask_id and i in stats] if kind == "whole canvas" else A
+        gaps = [stats[i].m1 - stats[i].m2 for i in pool]
+        if kind == "probability gap":
+            gaps = [stats[i].p1 - stats[i].p2 for i in pool]
+        stat = {"max": max, "min": min}.get(kind, lambda g: sum(g) / len(g))(gaps) if gaps else 0.0
+        ok = stat > p.gap_threshold if kind == "strict" else stat >= p.gap_threshold
+        E = list(A) if (A and ok) else []
+        if kind == "per token":
+            E = [i for i in A if stats[i].m1 - stats[i].m2 >= p.gap_threshold]
+        near = list(A) if A and abs(stat - p.gap_threshold) <= 1e-3 * abs(p.gap_threshold) else []
+        k = min(k_transfer, len(A))
+        U = sorted(sorted(A, key=lambda i: (-stats[i].p1, i))[:k])
+        for i in set(E) | set(U):
+            x[i] = stats[i].i1
+        return jo.StepReport(E, U, near, {}, {})
+    return fn
+
+
+GAP_MUTATIONS = ["max", "min", "strict", "whole canvas", "per token", "probability gap"]
+
+
+def test_gap_variant_without_a_mistake_passes():
+    import unittest.mock as um
+    with um.patch.object(jo, "accept_freeze", gap_variant("none")):
+        assert not some_pin_fails(GAP_PINS)
+
+
+@pytest.mark.parametrize("kind", GAP_MUTATIONS)
+def test_global_gap_pins_catch(kind, monkeypatch):
+    monkeypatch.setattr(jo, "accept_freeze", gap_variant(kind))
+    assert some_pin_fails(GAP_PINS), f"no pin noticed: {kind}"
 
 
 # ---------------------------------------------------------------- denoiser side
