@@ -50,17 +50,25 @@ int jot_last_cuda_error(void);
  * early-exit mask (Section 4.2 "Implementation details"); 1: it ranks only what early exit left.
  * gate: JOT_GATE_RATIO is the paper's test r >= tau (Eq. 8).  JOT_GATE_MAXPROB replaces it by the fixed
  * probability gate the paper contrasts JoT with (Section 2): p1 >= prob_threshold, no spatial modulation;
- * the transfer schedule and the OR are unchanged.  0 < prob_threshold <= 1 is required then, any other
- * gate value is refused (JOT_ERR_ARG). */
+ * the transfer schedule and the OR are unchanged.  0 < prob_threshold <= 1 is required then.
+ * JOT_GATE_GLOBAL_GAP is the global early-commit rule the paper contrasts JoT with (Section 2: once the top-2
+ * confidence gap exceeds a threshold, all remaining masked positions are finalised simultaneously), read as:
+ * the mean over the sequence's candidates (masked positions of the current block) of the top-2 logit gap
+ * top1 - top2 is compared with gap_threshold (inclusive, in fp32) and either every candidate exits or none
+ * does; schedule and OR unchanged.  The compared system stages three thresholds over decoding progress
+ * (7.5 / 5.0 / 2.5, Section 5.1): here the threshold is one input, which a caller stepping through
+ * jot_denoise_step / jot_accept_freeze may change from step to step.  Any other gate value is refused
+ * (JOT_ERR_ARG). */
 typedef struct {
     float tau_max, tau_min, gamma;
     int32_t D;
     float eps;
     int32_t schedule_after_exit;
-    int32_t gate;            /* 0 = JOT_GATE_RATIO, 1 = JOT_GATE_MAXPROB */
+    int32_t gate;            /* 0 = JOT_GATE_RATIO, 1 = JOT_GATE_MAXPROB, 2 = JOT_GATE_GLOBAL_GAP */
     float prob_threshold;    /* JOT_GATE_MAXPROB: finalise when p1 >= prob_threshold */
+    float gap_threshold;     /* JOT_GATE_GLOBAL_GAP: finalise every candidate when their mean top-2 logit gap >= this */
 } jot_params;
-enum { JOT_GATE_RATIO = 0, JOT_GATE_MAXPROB = 1 };
+enum { JOT_GATE_RATIO = 0, JOT_GATE_MAXPROB = 1, JOT_GATE_GLOBAL_GAP = 2 };
 
 /* Geometry of the denoiser f_theta (Algorithm 1 treats it as given).  Llama-style: RMSNorm,
  * rotate-half RoPE on absolute canvas positions, grouped-query attention without any mask, SwiGLU

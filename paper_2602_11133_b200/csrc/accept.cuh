@@ -19,8 +19,9 @@ struct AcceptParamsDev {     // mirrors jot_params
     int32_t D;
     float eps;
     int32_t schedule_after_exit;
-    int32_t gate;                // 0: ratio r >= tau (Eq. 8); 1: fixed probability gate p1 >= prob_threshold
-    float prob_threshold;
+    int32_t gate;                // 0: ratio r >= tau (Eq. 8); 1: fixed probability gate p1 >= prob_threshold;
+    float prob_threshold;        // 2: global early commit, mean top-2 logit gap of the candidates >= gap_threshold
+    float gap_threshold;
 };
 
 // Per-sequence loop state used by the generate loop (device resident).
@@ -72,7 +73,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     __shared__ float gpow[kMaxD + 1];
     __shared__ int n_cand_sh, warp_counts[kAcceptThreads / 32], n_final_sh;
     __shared__ float inv_wmax;
-    __shared__ float ratio_sums[kAcceptThreads / 32];
+    __shared__ float ratio_sums[kAcceptThreads / 32], gap_sums[kAcceptThreads / 32];
 
     const AcceptParamsDev prm = a.params ? a.params[a.per_seq_params ? b : 0] : a.uniform;
     int32_t* x = a.tokens + (size_t)b * L;
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     const int n_cand = n_cand_sh;
 
     // per candidate: ratio, threshold, early-exit decision
-    float r_sum = 0.f;
+    float r_sum = 0.f, gap_sum = 0.f;
     for (int c = tid; c < n_cand; c += blockDim.x) {
         const int i = cand[c];
         const size_t gi = (size_t)b * L + i;
@@ -152,9 +153,16 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
         const float tau = prm.tau_max - (prm.tau_max - prm.tau_min) * phi; // Eq. 7
         cand_S[c] = S;
         r_sum += r;
+        gap_sum += m1 - m2;
         // Eq. 8; or the fixed probability gate the paper contrasts it with (p1 = 1/S, no spatial modulation)
-        const bool exit_now = prm.gate == 1 ? (1.f / S >= prm.prob_threshold) : (r >= tau);
+        // (the global early-commit gate decides for all candidates together, after the sum below)
+        const bool exit_now = prm.gate == 1 ? (1.f / S >= prm.prob_threshold) : (prm.gate == 2 ? false : r >= tau);
         cand_flag[c] = exit_now ? 1 : 0;
+    }
+    if (prm.gate == 2) {                                       // fixed-order tree: the same sum on every run
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) gap_sum += __shfl_xor_sync(0xffffffffu, gap_sum, o);
+        if ((tid & 31) == 0) gap_sums[tid >> 5] = gap_sum;
     }
     if (a.mean_ratio) {                                        // fixed-order tree: the same sum on every run
 #pragma unroll
@@ -162,6 +170,14 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
         if ((tid & 31) == 0) ratio_sums[tid >> 5] = r_sum;
     }
     __syncthreads();
+    if (prm.gate == 2 && n_cand > 0) {
+        // global early commit: every candidate exits when the mean top-2 logit gap clears the threshold
+        float t = 0.f;
+        for (int w = 0; w < kAcceptThreads / 32; ++w) t += gap_sums[w];
+        if (t / (float)n_cand >= prm.gap_threshold)
+            for (int c = tid; c < n_cand; c += blockDim.x) cand_flag[c] = 1;
+    }
+    if (prm.gate == 2) __syncthreads();                        // the schedule below may read other threads' flags
 
     // transfer schedule: the k candidates with the largest p1 = 1/S, i.e. the smallest S; equal S
     // resolves to the lower position.  Rank by counting (candidate lists are short).

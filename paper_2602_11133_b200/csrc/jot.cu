@@ -665,6 +665,7 @@ int launch_accept(const AcceptArgs& a, cudaStream_t st) {
 bool params_ok(const jot_params* p) {
     if (!p || p->D < 1 || p->D > kMaxD) return false;
     if (p->gate == JOT_GATE_MAXPROB) return p->prob_threshold > 0.f && p->prob_threshold <= 1.f;
+    if (p->gate == JOT_GATE_GLOBAL_GAP) return p->gap_threshold == p->gap_threshold;      // anything but NaN
     return p->gate == JOT_GATE_RATIO;
 }
 
@@ -909,7 +910,7 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
     cudaStream_t st = (cudaStream_t)stream;
     AcceptArgs a{};
     a.uniform = AcceptParamsDev{params->tau_max, params->tau_min, params->gamma, params->D, params->eps,
-                                params->schedule_after_exit, params->gate, params->prob_threshold};
+                                params->schedule_after_exit, params->gate, params->prob_threshold, params->gap_threshold};
     a.params = nullptr;
     a.mask_id = mask_id; a.tokens = d_tokens; a.B = B; a.L = L;
     a.blk_lo = blk_lo; a.blk_hi = blk_hi; a.k_transfer = k_transfer;

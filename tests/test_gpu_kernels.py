@@ -314,6 +314,39 @@ def test_lm_head_sampling_low_temperature_is_argmax(jot):
     model.close()
 
 
+@pytest.mark.parametrize("B,L,P,lo,hi,k", [(4, 384, 128, 128, 384, 1), (2, 1000, 10, 10, 1000, 7), (6, 704, 192, 224, 256, 1)])
+def test_accept_freeze_global_gap_gate_matches_oracle(jot, B, L, P, lo, hi, k):
+    """The global early-commit rule the paper contrasts JoT with (Section 2): per sequence, all candidates exit
+    when their mean top-2 logit gap clears the threshold, else none; schedule and OR unchanged.  The threshold is
+    set at the median of the sequences' mean gaps so that both outcomes occur."""
+    V, mask_id = 5000, 4321
+    tokens, top1, top2, sumexp, argmax = random_accept_case(B * 31 + L, B, L, P, mask_id, V)
+    means = []
+    for b in range(B):
+        c = [i for i in range(lo, hi) if tokens[b, i] == mask_id]
+        means.append(float(np.mean([float(top1[b, i]) - float(top2[b, i]) for i in c])))
+    thr = float(np.median(means)) * 1.0001 + 1e-4
+    params = jo.JotParams(gate="globalgap", gap_threshold=thr)
+    want, reps = oracle_accept_batch(torch.from_numpy(tokens), top1, top2, sumexp, argmax, params, mask_id, lo, hi, k)
+    d_tok = torch.from_numpy(tokens).cuda()
+    st = jot.Stats(*[torch.from_numpy(t).cuda() for t in (top1, top2, sumexp, argmax)])
+    reason = torch.zeros(B, L, dtype=torch.uint8, device="cuda")
+    jot.accept_freeze(jot.Params(gate=jot.GATE_GLOBAL_GAP, gap_threshold=thr), mask_id, d_tok, lo, hi, k, st, exit_reason=reason)
+    got = d_tok.cpu()
+    outcomes = set()
+    for b in range(B):
+        assert not reps[b].near_margin, "the case should not sit on the threshold"
+        outcomes.add(len(reps[b].exited) > 0)
+        assert torch.equal(got[b], want[b]), b
+        n_cand = sum(1 for i in range(lo, hi) if tokens[b, i] == mask_id)
+        assert len(reps[b].exited) in (0, n_cand)                 # everything or nothing
+        flagged = int((reason[b].cpu() & 1).sum())
+        assert flagged == len(reps[b].exited)
+    assert outcomes == {True, False}
+    with pytest.raises(jot.JotError):
+        jot.accept_freeze(jot.Params(gate=jot.GATE_GLOBAL_GAP, gap_threshold=float("nan")), mask_id, d_tok, lo, hi, k, st)
+
+
 @pytest.mark.parametrize("B,L,P,lo,hi,k", [(4, 384, 128, 128, 384, 1), (2, 1000, 10, 10, 1000, 7), (3, 704, 192, 224, 256, 1)])
 @pytest.mark.parametrize("pth", [0.5, 0.9])
 def test_accept_freeze_probability_gate_matches_oracle(jot, B, L, P, lo, hi, k, pth):
@@ -345,6 +378,6 @@ def test_accept_freeze_probability_gate_matches_oracle(jot, B, L, P, lo, hi, k, 
     jot.accept_freeze(jot.Params(90, 1, 0.5, 8), mask_id, t2, lo, hi, k, st)
     assert not torch.equal(t2, d_tok)
     with pytest.raises(jot.JotError):
-        jot.accept_freeze(jot.Params(gate=2), mask_id, t2, lo, hi, k, st)
+        jot.accept_freeze(jot.Params(gate=3), mask_id, t2, lo, hi, k, st)
     with pytest.raises(jot.JotError):
         jot.accept_freeze(jot.Params(gate=jot.GATE_MAXPROB, prob_threshold=0.0), mask_id, t2, lo, hi, k, st)

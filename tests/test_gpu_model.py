@@ -358,3 +358,49 @@ def test_generation_trace_matches_oracle(jot):
         assert torch.equal(t2.mean_ratio[:, 0], trace.mean_ratio[:, 0])
         assert torch.equal(t2.n_candidates[:, 0], trace.n_candidates[:, 0])
     model.close()
+
+
+def test_generation_under_the_global_early_commit_gate(jot):
+    """The global early-commit rule (Section 2) inside Algorithm 1 on the tiny model with the planted bump:
+    a threshold nothing clears gives plain schedule decoding (T steps), one everything clears commits a block
+    per step, and a threshold in between reproduces the oracle's trajectory (tokens and step count)."""
+    g = inputs.TINY
+    P, G, T, Lb = 32, 64, 64, 16
+    w_cpu = inputs.model_weights(g, seed=0)
+    w_gpu = inputs.weights_to(w_cpu, "cuda")
+    prompt = inputs.prompt(0, 1, P, g.vocab, g.mask_id)
+    bump = inputs.logit_bump(9, 1, P + G, g.vocab, g.mask_id, hi=12.0)
+    d_bump = dict(bump_id=bump[0].cuda(), bump_val=bump[1].cuda())
+    model = jot.Model(g, w_gpu, 1, P + G)
+    _, used, _ = model.generate(prompt.cuda(), G, T, jot.Params(gate=jot.GATE_GLOBAL_GAP, gap_threshold=1e30), Lb, **d_bump)
+    assert used[0] == T
+    out, used, _ = model.generate(prompt.cuda(), G, T, jot.Params(gate=jot.GATE_GLOBAL_GAP, gap_threshold=-1e30), Lb, **d_bump)
+    assert used[0] == G // Lb and (out != g.mask_id).all()
+    # the blocks' mean gaps differ (random bumps): a threshold between them commits some blocks at once and leaves
+    # the others to the schedule
+    for thr in (4.0, 4.5, 5.0, 5.5, 6.0, 6.5, 7.0, 8.0):
+        tr = oracle_trajectory(g, w_cpu, prompt[0].tolist(), G, T, jo.JotParams(gate="globalgap", gap_threshold=thr), Lb, bump)
+        if G // Lb < tr.steps_used < T:
+            break
+    assert G // Lb < tr.steps_used < T                      # the gate fired somewhere, but not everywhere
+    out, used, _ = model.generate(prompt.cuda(), G, T, jot.Params(gate=jot.GATE_GLOBAL_GAP, gap_threshold=thr), Lb, **d_bump)
+    # the mean gap of a step is within the logit tolerance of the oracle's; a step whose mean sits that close to
+    # the threshold may legitimately go either way, every other step must agree
+    # (2-layer model: the measured logit error is ~2e-3, so 0.02 on a mean of gaps is a wide berth)
+    margins = [abs(float(np.mean(gaps)) - thr) for gaps in step_gaps(tr, g, w_cpu, bump)]
+    print(f"threshold {thr}: oracle used {tr.steps_used} steps, smallest |mean gap - threshold| {min(margins):.3f}")
+    if min(margins) >= 0.02:
+        assert used[0] == tr.steps_used and out.cpu()[0].tolist() == tr.x
+    model.close()
+
+
+def step_gaps(tr, g, w_cpu, bump):
+    """Top-2 logit gaps of the candidates at every step of an oracle trajectory."""
+    out = []
+    for x, (lo, hi) in zip(tr.canvases, tr.blocks):
+        rows = [i for i in range(lo, hi) if x[i] == g.mask_id]
+        l = mo.logits(g, w_cpu, torch.tensor([x], dtype=torch.int32), rows=[(0, i) for i in rows])
+        for r, i in enumerate(rows):
+            l[r, int(bump[0][0, i])] += float(bump[1][0, i])
+        out.append([float(st.m1 - st.m2) for st in (jo.row_stats(l[r].numpy(), g.mask_id) for r in range(len(rows)))])
+    return out
