@@ -72,7 +72,8 @@ struct GemmSmem {
     static constexpr int B_BYTES = BN * kBK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = (BN == 256) ? JOT_GEMM_STAGES_256 : JOT_GEMM_STAGES_128;
-    static constexpr int DYN_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align to 1024
+    static constexpr int STAGING_BYTES = 4 * 32 * 36 * 4;          // per epilogue warp 32 x 36 floats (EPI_PARTIAL)
+    static constexpr int DYN_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024;   // + slack to align to 1024
 };
 
 // How the stats kernel splits the vocabulary: row blocks run side by side over the same vocabulary
@@ -124,7 +125,7 @@ __device__ __forceinline__ void stats_row_init(const GemmParams& p, int row, Sta
 // it 32 columns at a time from tensor memory at `t_acc`.  Shared by the one-CTA and the CTA-pair kernels.
 template <int BN, int EPI>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_acc, int row, int n_blk, int ks,
-                                              int n_out, StatsRow& st) {
+                                              int n_out, StatsRow& st, float* stg = nullptr) {
     constexpr float L2E = 1.4426950408889634f;
     (void)L2E; (void)ks; (void)n_out; (void)st;
     if (EPI == EPI_STORE) {
@@ -220,20 +221,32 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
             }
         }
     } else if (EPI == EPI_PARTIAL) {
+        // A thread owns a row, so its 32 columns are 128 contiguous bytes, but a warp's rows lie N * 4 bytes
+        // apart.  The warp turns its 32 x 32 block around through `stg` (rows padded to 36 floats: no bank
+        // conflicts either way) so that every store instruction covers four whole 128-byte lines.
+        const int lane = threadIdx.x & 31;
+        const int row0 = row - lane;                          // first row of this warp's block
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
             float v[32];
             tmem_ld32(t_acc + c * 32, v);
             tmem_ld_wait();
             const int col0 = n_blk * BN + c * 32;
-            if (row < p.M) {
-                float* dst = p.partial + ((size_t)ks * p.M + row) * p.N + col0;
 #pragma unroll
-                for (int g = 0; g < 8; ++g)
-                    if (col0 + g * 4 < p.N)           // N is a multiple of 8
-                        *reinterpret_cast<float4*>(dst + g * 4) =
-                            make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+            for (int g = 0; g < 8; ++g)
+                *reinterpret_cast<float4*>(stg + lane * 36 + g * 4) = make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+            __syncwarp();
+            const int cg = lane & 7;                          // four columns of the row
+            if (col0 + cg * 4 < p.N) {                        // N is a multiple of 8
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int r = it * 4 + (lane >> 3);
+                    if (row0 + r < p.M)
+                        *reinterpret_cast<float4*>(p.partial + ((size_t)ks * p.M + row0 + r) * p.N + col0 + cg * 4) =
+                            *reinterpret_cast<const float4*>(stg + r * 36 + cg * 4);
+                }
             }
+            __syncwarp();
         }
     } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
@@ -480,7 +493,8 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
             tc_fence_after();
-            epilogue_tile<BN, EPI>(p, lane_base + acc * BN, m_blk * kBM + row_in_tile, n_blk, ks, n_out, st);
+            epilogue_tile<BN, EPI>(p, lane_base + acc * BN, m_blk * kBM + row_in_tile, n_blk, ks, n_out, st,
+                                   reinterpret_cast<float*>(smem + STAGES * SM::STAGE_BYTES) + quad * (32 * 36));
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
