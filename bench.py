@@ -39,7 +39,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, keyed by kernel class and workload; removed (-> null) whenever the kernel changes afterwards.
 NCU_TRAFFIC = {
-    ("llada8b", "gemm_gate_up"): 215.4e6,     # profiles/gemm_llada8b_m384.md
+    ("llada8b", "gemm_gate_up"): 216.7e6,     # profiles/gemm_llada8b_m384.md
     ("lmhead", "lm_head"): 1067.0e6,          # profiles/lm_head_pair_lmhead.md
 }
 
