@@ -276,6 +276,43 @@ def test_generate_threshold_zero_finishes_one_step_per_block():
     assert 32 / tr.steps_used == 8.0
 
 
+def test_generate_decodes_blocks_left_to_right():
+    # Semi-autoregressive decoding (Appendix "Experimental Configuration": the canvas is generated "in fixed-size
+    # blocks", each block only after the ones before it): a stub model that writes, for every position, whether the
+    # position one block to its LEFT was already resolved when it was asked.  Left to right, every block after
+    # the first sees a resolved left neighbour and a masked right one; any other order changes the tokens.
+    P, Lb, nb = 4, 4, 4
+    G = Lb * nb
+    asked = []
+
+    def stats_fn(x, A):
+        asked.append((min(A), max(A)))
+        out = {}
+        for i in A:
+            left_resolved = x[i - Lb] != M                       # prompt or an earlier block
+            right_masked = i + Lb >= len(x) or x[i + Lb] == M
+            tok = 100 + (1 if left_resolved else 0) + (2 if right_masked else 0)
+            out[i] = jo.RowStats(5.0, tok, 0.0, 1.5)
+        return out
+    tr = jo.generate(None, [1, 2, 3, 4], G, G, jo.JotParams(0.0, 0.0, 0.5, 8), M, Lb, stats_fn=stats_fn)
+    assert tr.x[P:] == [103] * G                                 # left resolved AND right still masked, everywhere
+    assert tr.blocks == [(P + b * Lb, P + (b + 1) * Lb) for b in range(nb)]
+    assert asked == [(P + b * Lb, P + (b + 1) * Lb - 1) for b in range(nb)]
+    # one block at a time: a step never touches a position outside the block it was run for
+    for cv, nxt, (lo, hi) in zip(tr.canvases, tr.canvases[1:] + [tr.x], tr.blocks):
+        assert all(a == b for i, (a, b) in enumerate(zip(cv, nxt)) if not lo <= i < hi)
+
+
+def test_generate_schedule_table_restarts_in_every_block():
+    # Nothing clears the gate, so each step finalises exactly what the schedule reveals: 6 positions over the 4
+    # steps of a block are 2, 2, 1, 1 (the remainder goes to the earliest steps), and the next block starts over.
+    inf = float("inf")
+    tr = jo.generate(None, [7, 8], 12, 8, jo.JotParams(inf, inf, 0.5, 8), M, 6, stats_fn=random_stats_fn(3))
+    assert tr.steps_used == 8
+    assert [len(r.scheduled) for r in tr.reports] == [2, 2, 1, 1, 2, 2, 1, 1]
+    assert [cv.count(M) for cv in tr.canvases] == [12, 10, 8, 7, 6, 4, 2, 1]
+
+
 def test_generate_with_logits_fn_excludes_mask_token():
     V = 12
     mid = V - 1

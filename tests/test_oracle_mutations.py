@@ -168,6 +168,35 @@ def test_decision_pins_catch(name, monkeypatch):
     assert some_pin_fails(ACCEPT_PINS), f"no pin noticed: {name}"
 
 
+def generate_variant(old, new):
+    """jo.generate with one line of its source replaced (the planted mistake), compiled in the oracle's namespace."""
+    import inspect
+    src = inspect.getsource(jo.generate)
+    assert src.count(old) == 1, old
+    ns = dict(vars(jo))
+    exec(src.replace(old, new), ns)
+    return ns["generate"]
+
+
+LOOP_MUTATIONS = {
+    "blocks decoded right to left": ("for blk in range(nb):", "for blk in reversed(range(nb)):"),
+    "blocks decoded from the second one on, the first last": (
+        "for blk in range(nb):", "for blk in list(range(1, nb)) + [0]:"),
+    "candidates are every masked position, not the current block's": (
+        "A = [i for i in range(lo, hi) if x[i] == mask_id]             # M_n",
+        "A = [i for i in range(P, len(x)) if x[i] == mask_id]"),
+    "the schedule table restarts only once": ("rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[s],",
+                                              "rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[min(traj.steps_used, Tb - 1)],"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(LOOP_MUTATIONS))
+def test_loop_pins_catch(name, monkeypatch):
+    old, new = LOOP_MUTATIONS[name]
+    monkeypatch.setattr(jo, "generate", generate_variant(old, new))
+    assert some_pin_fails(ACCEPT_PINS), f"no pin noticed: {name}"
+
+
 def gap_variant(kind):
     """accept_freeze whose global early-commit branch carries one planted mistake."""
     orig = jo.accept_freeze
