@@ -64,6 +64,8 @@ struct GemmParams {
     int step_value;               // step_value); b = flat canvas index / L
     float2* partials2;            // [chunks][R_pad] (best perturbed score, bitcast token)
     int R_pad;                    // row capacity of one chunk of partials (multiple of 128)
+    // slab kernel only (gemm_slab.cuh): first pair-slab of the launch and pairs per cluster (K ranges)
+    int slab0, slab_split;
 };
 
 template <int BN>
@@ -425,17 +427,18 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     };
 
     if (warp == 0) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            int m_blk, n_blk;
-            bool ok = true;
-            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
-                    uint8_t* sA = smem + stage * SM::STAGE_BYTES;
-                    uint8_t* sB = sA + SM::A_BYTES;
+        // ================= TMA producer (the whole warp runs the loop, one lane issues) =================
+        const bool elected = elect_one();
+        int stage = 0;
+        uint32_t phase = 0;
+        int m_blk, n_blk;
+        bool ok = true;
+        for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
+                uint8_t* sA = smem + stage * SM::STAGE_BYTES;
+                uint8_t* sB = sA + SM::A_BYTES;
+                if (elected) {
                     mbar_arrive_expect_tx(&full_bar[stage], SM::STAGE_BYTES);
                     tma_load_2d(sA, &tmA, &full_bar[stage], kb * kBK, m_blk * kBM);
                     if (EPI == EPI_SWIGLU) {
@@ -446,39 +449,49 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
                     } else {
                         tma_load_2d(sB, &tmB, &full_bar[stage], kb * kBK, n_blk * BN);
                     }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
-            int stage = 0, acc = 0;
-            uint32_t phase = 0, acc_phase = 0;
-            int m_blk, n_blk;
-            bool ok = true;
-            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
-                if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abortp)) break;
+        // ================= MMA issuer (the whole warp runs the loop, one lane issues) =================
+        // The operand descriptors of a stage differ from stage 0's only in the 16-byte-granular address field
+        // and are advanced by additions (the field never carries: shared-memory addresses stay below 256 KB).
+        const bool elected = elect_one();
+        const uint64_t ad0 = umma_desc_k128(smem_u32(smem));
+        const uint64_t bd0 = ad0 + (SM::A_BYTES >> 4);
+        constexpr uint32_t STAGE_UNITS = SM::STAGE_BYTES >> 4;
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        uint64_t ad = ad0, bd = bd0;
+        int m_blk, n_blk;
+        bool ok = true;
+        for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+            if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abortp)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * BN;
+            uint32_t accum = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = smem_u32(smem + stage * SM::STAGE_BYTES);
-                    const uint32_t b_addr = a_addr + SM::A_BYTES;
+                if (elected) {
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k) {
-                        umma_bf16(d_tmem, umma_desc_k128(a_addr + k * 32), umma_desc_k128(b_addr + k * 32), IDESC,
-                                  (kb > kb0) || (k != 0));
-                    }
+                    for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, ad + 2 * k, bd + 2 * k, IDESC, accum | k);
                     umma_commit(&empty_bar[stage]);       // smem stage reusable once these MMAs retire
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (!ok) break;
-                umma_commit(&acc_full[acc]);              // accumulator complete
-                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                __syncwarp();
+                accum = 1;
+                ad += STAGE_UNITS;
+                bd += STAGE_UNITS;
+                if (++stage == STAGES) { stage = 0; phase ^= 1; ad = ad0; bd = bd0; }
             }
+            if (!ok) break;
+            if (elected) umma_commit(&acc_full[acc]);     // accumulator complete
+            __syncwarp();
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+        __syncwarp();
     } else {
         // ================= epilogue (warps 2..5) =================
         const int quad = warp & 3;                        // TMEM lanes [32*quad, 32*quad+32)

@@ -111,57 +111,71 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
     };
 
     if (warp == 0) {
-        // ================= TMA producer (both CTAs) =================
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            int m_blk, n_blk;
-            bool ok = true;
-            for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
-                // this CTA's half of the W tile: SwiGLU pairs 128 gate rows (leader) with the matching 128 up rows
-                const int w_row = (EPI == EPI_SWIGLU) ? (rank == 0 ? n_blk * kBM : p.N / 2 + n_blk * kBM)
-                                                      : n_blk * BN + rank * kBM;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
-                    uint8_t* sA = smem + stage * kPairStageBytes;
-                    uint8_t* sB = sA + HALF_BYTES;
-                    const uint32_t full_leader = mapa_u32(&full_bar[stage], 0);
+        // ================= TMA producer (both CTAs; the whole warp runs the loop, one lane issues) =================
+        const bool elected = elect_one();
+        int stage = 0;
+        uint32_t phase = 0;
+        int m_blk, n_blk;
+        bool ok = true;
+        for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
+            // this CTA's half of the W tile: SwiGLU pairs 128 gate rows (leader) with the matching 128 up rows
+            const int w_row = (EPI == EPI_SWIGLU) ? (rank == 0 ? n_blk * kBM : p.N / 2 + n_blk * kBM)
+                                                  : n_blk * BN + rank * kBM;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
+                uint8_t* sA = smem + stage * kPairStageBytes;
+                uint8_t* sB = sA + HALF_BYTES;
+                const uint32_t full_leader = mapa_u32(&full_bar[stage], 0);
+                if (elected) {
                     if (leader) mbar_arrive_expect_tx(&full_bar[stage], 2 * kPairStageBytes);
                     tma_load_2d_pair(sA, &tmA, full_leader, kb * kBK, m_blk * kBM);
                     tma_load_2d_pair(sB, &tmB, full_leader, kb * kBK, w_row);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer (leader CTA only) =================
-        if (lane == 0 && leader) {
+        // ================= MMA issuer (leader CTA only; the whole warp runs the loop, one lane issues) ==========
+        // One thread issues every MMA of the pair, so the loop is kept to a few instructions per MMA: the operand
+        // descriptors of a stage differ from stage 0's only in the 16-byte-granular address field and are
+        // advanced by additions (the field never carries: shared-memory addresses stay below 256 KB).
+        if (leader) {
+            const bool elected = elect_one();
+            const uint64_t ad0 = umma_desc_k128(smem_u32(smem));
+            const uint64_t bd0 = ad0 + (HALF_BYTES >> 4);
+            constexpr uint32_t STAGE_UNITS = kPairStageBytes >> 4;
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
+            uint64_t ad = ad0, bd = bd0;
             int m_blk, n_blk;
             bool ok = true;
             for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
                 if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abortp)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
+                uint32_t accum = 0;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(smem + stage * kPairStageBytes);
-                    const uint32_t b_addr = a_addr + HALF_BYTES;
+                    if (elected) {
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k) {
-                        umma_bf16_pair(d_tmem, umma_desc_k128(a_addr + k * 32), umma_desc_k128(b_addr + k * 32), IDESC,
-                                       (kb | k) != 0);
+                        for (int k = 0; k < kBK / 16; ++k) umma_bf16_pair(d_tmem, ad + 2 * k, bd + 2 * k, IDESC, accum | k);
+                        umma_commit_pair(&empty_bar[stage], 0x3);     // both CTAs may refill this stage
                     }
-                    umma_commit_pair(&empty_bar[stage], 0x3);     // both CTAs may refill this stage
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    __syncwarp();
+                    accum = 1;
+                    ad += STAGE_UNITS;
+                    bd += STAGE_UNITS;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; ad = ad0; bd = bd0; }
                 }
                 if (!ok) break;
-                umma_commit_pair(&acc_full[acc], 0x3);            // both CTAs' accumulators are complete
+                if (elected) umma_commit_pair(&acc_full[acc], 0x3);   // both CTAs' accumulators are complete
+                __syncwarp();
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
         }
+        __syncwarp();
     } else {
         // ================= epilogue (warps 2..5, both CTAs) =================
         const int quad = warp & 3;

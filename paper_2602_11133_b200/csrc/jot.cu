@@ -19,6 +19,7 @@
 #include "attention.cuh"
 #include "gemm.cuh"
 #include "gemm2.cuh"
+#include "gemm_slab.cuh"
 #include "glue.cuh"
 
 using namespace jot;
@@ -158,6 +159,120 @@ int launch_pair_t(const GemmParams& p, const CUtensorMap& tmA, const CUtensorMap
     return launch_check();
 }
 
+struct WeightMaps {     // one weight matrix as B operand, for both tile widths
+    CUtensorMap m128, m256;
+};
+
+int make_weight_maps(const DeviceInfo* di, WeightMaps* w, const void* ptr, int rows, int cols, bool swiglu) {
+    // swiglu tiles fetch gate and up rows as two boxes of half the tile width
+    JOT_TRY(make_map_2d(di, &w->m128, ptr, rows, cols, cols, swiglu ? 64 : 128));
+    JOT_TRY(make_map_2d(di, &w->m256, ptr, rows, cols, cols, swiglu ? 128 : 256));
+    return JOT_OK;
+}
+
+// ---------------------------------------------------------------- slab kernel (canvases of at most 512 rows)
+// A token matrix [M, K] as the slab kernel's N operand: one box shape per accumulator (half its tokens).
+struct SlabMaps {
+    CUtensorMap x0, x1;
+};
+int make_slab_maps(const DeviceInfo* di, SlabMaps* sm, const void* ptr, int M, int K, int ld) {
+    const SlabGeom g = slab_geom(M, 1);
+    JOT_TRY(make_map_2d(di, &sm->x0, ptr, M, K, ld, (uint32_t)(g.n0 / 2)));
+    JOT_TRY(make_map_2d(di, &sm->x1, ptr, M, K, ld, (uint32_t)(g.n1 ? g.n1 / 2 : g.n0 / 2)));
+    return JOT_OK;
+}
+
+// Clusters of `split` CTA pairs; the launch covers pair-slabs slab0 .. slab0 + n_slabs - 1.
+template <int EPI>
+int launch_slab_t(GemmParams p, const CUtensorMap& tmW, const SlabMaps& tmX, int slab0, int n_slabs, int split,
+                  cudaStream_t st) {
+    static thread_local bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev & 63]) {
+        JOT_CUDA(cudaFuncSetAttribute(gemm_slab_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSlabMaxSmem));
+        attr_set[dev & 63] = true;
+    }
+    p.slab0 = slab0;
+    p.slab_split = split;
+    const SlabGeom g = slab_geom(p.M, split);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(n_slabs * 2 * split));
+    cfg.blockDim = dim3(kSlabThreads);
+    cfg.dynamicSmemBytes = (size_t)g.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)(2 * split);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaLaunchKernelEx(&cfg, gemm_slab_kernel<EPI>, p, tmW, tmX.x0, tmX.x1);
+    return launch_check();
+}
+
+// How many clusters of `split` pairs the device runs side by side (1 CTA per SM: the kernel takes all shared memory).
+int slab_cluster_capacity(int sms, int split) {
+    static thread_local int cap[64][5] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int& c = cap[dev & 63][split];
+    if (c == 0) {
+        cudaFuncSetAttribute(gemm_slab_kernel<SLAB_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSlabMaxSmem);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * split * 64));
+        cfg.blockDim = dim3(kSlabThreads);
+        cfg.dynamicSmemBytes = (size_t)kSlabMaxSmem - 1024;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)(2 * split);
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_slab_kernel<SLAB_STORE>, &cfg) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = sms / (2 * split) * 3 / 4;          // a guess that errs on the low side
+        }
+        c = n > 0 ? n : 1;
+    }
+    return c;
+}
+
+// Largest K split (pairs per cluster) that keeps `n_slabs` clusters in one wave, leaves every pair at least 8
+// k-blocks and fits the reduce-scatter buffers in shared memory.
+int slab_pick_split(int M, int n_slabs, int num_kb, int sms) {
+    for (int s = 4; s > 1; --s) {
+        if (num_kb / s < 8) continue;
+        if (slab_geom(M, s).smem_bytes > kSlabMaxSmem) continue;
+        if (n_slabs <= slab_cluster_capacity(sms, s)) return s;
+    }
+    return 1;
+}
+
+int run_slab(const DeviceInfo* di, const SlabMaps& tmX, const WeightMaps& w, int epi, const GemmParams& p, cudaStream_t st) {
+    const int n_out = (epi == EPI_SWIGLU) ? p.N / 2 : p.N;
+    const int per_slab = (epi == EPI_SWIGLU) ? 128 : 256;                 // output features per CTA pair
+    const int n_slabs = (n_out + per_slab - 1) / per_slab;
+    const int num_kb = (p.K + kBK - 1) / kBK;
+    auto go = [&](int slab0, int n, int split) -> int {
+        if (n <= 0) return JOT_OK;
+        if (epi == EPI_STORE) return launch_slab_t<SLAB_STORE>(p, w.m128, tmX, slab0, n, split, st);
+        if (epi == EPI_QKV) return launch_slab_t<SLAB_QKV>(p, w.m128, tmX, slab0, n, split, st);
+        return launch_slab_t<SLAB_SWIGLU>(p, w.m128, tmX, slab0, n, split, st);
+    };
+    const int cap1 = slab_cluster_capacity(di->sms, 1);
+    // whole waves of unsplit slabs first; what is left over (or a projection with few slabs) is cut along K so
+    // that it still fills the machine
+    const int full = n_slabs / cap1 * cap1, rest = n_slabs - full;
+    JOT_TRY(go(0, full, 1));
+    return go(full, rest, slab_pick_split(p.M, rest, num_kb, di->sms));
+}
+
 // Which kernel shape moves the fewest operand bytes through an SM for this projection: waves x bytes per
 // k-block (48 KB for a 128 x 256 tile, 32 KB for a 128 x 128 tile, 32 KB per CTA of a 256 x 256 pair tile).
 enum { SHAPE_256 = 0, SHAPE_128 = 1, SHAPE_PAIR = 2 };
@@ -169,17 +284,6 @@ int pick_shape(int M, int n_out, int sms, bool allow_128) {
     const long cpair = m_blks >= 2 ? waves(((m_blks + 1) / 2) * n256, sms / 2) * 32 : (1L << 60);
     if (c256 <= c128 && c256 <= cpair) return SHAPE_256;
     return cpair <= c128 ? SHAPE_PAIR : SHAPE_128;
-}
-
-struct WeightMaps {     // one weight matrix as B operand, for both tile widths
-    CUtensorMap m128, m256;
-};
-
-int make_weight_maps(const DeviceInfo* di, WeightMaps* w, const void* ptr, int rows, int cols, bool swiglu) {
-    // swiglu tiles fetch gate and up rows as two boxes of half the tile width
-    JOT_TRY(make_map_2d(di, &w->m128, ptr, rows, cols, cols, swiglu ? 64 : 128));
-    JOT_TRY(make_map_2d(di, &w->m256, ptr, rows, cols, cols, swiglu ? 128 : 256));
-    return JOT_OK;
 }
 
 // Split-K factor for a plain projection: when 256-wide tiles leave most SMs idle, cut K into up to 4
@@ -203,7 +307,10 @@ struct NormAfter {
 };
 
 int run_gemm(const DeviceInfo* di, const CUtensorMap& tmA, const WeightMaps& w, int epi, GemmParams p, cudaStream_t st,
-             float* scratch = nullptr, size_t scratch_bytes = 0, NormAfter* norm = nullptr) {
+             float* scratch = nullptr, size_t scratch_bytes = 0, NormAfter* norm = nullptr,
+             const SlabMaps* tmX_slab = nullptr) {
+    // small canvases: weight rows as the MMA's M side, every token in tensor memory (gemm_slab.cuh)
+    if (tmX_slab && p.M <= kSlabMaxTokens) return run_slab(di, *tmX_slab, w, epi, p, st);      // callers decide when
     if (epi == EPI_STORE && scratch) {
         const int split = pick_split(p.M, p.N, p.K, di->sms, scratch_bytes);
         if (split > 1) {
@@ -299,7 +406,8 @@ struct jot_model {
     CUtensorMap tm_hsel, tm_qkv3, tm_vt;
     // A-operand maps of the projections for a pass over M rows (rows past M read as zero without memory
     // traffic): one set for the whole canvas, one for the rows of a block
-    struct ActMaps { int M = -1; CUtensorMap a, attn, act; };
+    // (x*: the same buffers as the token operand of the slab kernel, boxes of half an accumulator's tokens)
+    struct ActMaps { int M = -1; bool slab = false; CUtensorMap a, attn, act; SlabMaps xa, xattn, xact; };
     ActMaps maps_full, maps_span;
     // block-wise KV cache (caller's memory, optional): per layer the rotated Q/K rows and V^T of the whole canvas
     uint8_t* kv_base = nullptr;
@@ -427,6 +535,12 @@ int encode_act_maps(jot_model* m, jot_model::ActMaps* am, int M) {
     JOT_TRY(make_map_2d(m->di, &am->a, m->a, M, c.d_model, c.d_model, 128));
     JOT_TRY(make_map_2d(m->di, &am->attn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim, 128));
     JOT_TRY(make_map_2d(m->di, &am->act, m->act, M, c.d_ff, c.d_ff, 128));
+    am->slab = M <= kSlabPreferTokens;
+    if (am->slab) {
+        JOT_TRY(make_slab_maps(m->di, &am->xa, m->a, M, c.d_model, c.d_model));
+        JOT_TRY(make_slab_maps(m->di, &am->xattn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim));
+        JOT_TRY(make_slab_maps(m->di, &am->xact, m->act, M, c.d_ff, c.d_ff));
+    }
     am->M = M;
     return JOT_OK;
 }
@@ -497,7 +611,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
             ProfScope ps(m, JOT_PROF_GEMM_QKV, st);
             p.vt = cached ? m->kv_vt[l] : m->vt; p.rope_cs = m->rope_cs; p.L = L; p.Lp = Lp; p.nq = nq; p.nkv = nkv;
             p.hd = hd; p.rows_per_seq = Lr; p.pos0 = pos0;
-            JOT_TRY(run_gemm(m->di, am.a, m->wqkv[l], EPI_QKV, p, st));
+            JOT_TRY(run_gemm(m->di, am.a, m->wqkv[l], EPI_QKV, p, st, nullptr, 0, nullptr, am.slab ? &am.xa : nullptr));
         }
         AttnParams ap{};
         ap.B = B; ap.L = L; ap.nq = nq; ap.nkv = nkv; ap.out = m->attn; ap.status = status;
@@ -517,7 +631,8 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         {
             ProfScope ps(m, JOT_PROF_GEMM_O, st);
             NormAfter na{m->mlp_norm[l], m->a, c.rms_eps, false};
-            JOT_TRY(run_gemm(m->di, am.attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes, &na));
+            JOT_TRY(run_gemm(m->di, am.attn, m->wo[l], EPI_STORE, p, st, m->splitk, kSplitKBytes, &na,
+                             am.slab ? &am.xattn : nullptr));
             norm_ready = na.done;
         }
         if (!norm_ready) {
@@ -529,7 +644,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
         p.M = M; p.N = 2 * c.d_ff; p.K = d; p.C = m->act; p.ldc = c.d_ff; p.status = status;
         {
             ProfScope ps(m, JOT_PROF_GEMM_GATE_UP, st);
-            JOT_TRY(run_gemm(m->di, am.a, m->wgu[l], EPI_SWIGLU, p, st));
+            JOT_TRY(run_gemm(m->di, am.a, m->wgu[l], EPI_SWIGLU, p, st, nullptr, 0, nullptr, am.slab ? &am.xa : nullptr));
         }
         p = GemmParams{};
         p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
@@ -537,7 +652,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
             ProfScope ps(m, JOT_PROF_GEMM_DOWN, st);
             NormAfter na{l + 1 < c.n_layers ? m->attn_norm[l + 1] : nullptr, m->a, c.rms_eps, false};
             JOT_TRY(run_gemm(m->di, am.act, m->wdown[l], EPI_STORE, p, st, m->splitk, kSplitKBytes,
-                             na.gain ? &na : nullptr));
+                             na.gain ? &na : nullptr, am.slab ? &am.xact : nullptr));
             norm_ready = na.done;
         }
     }
@@ -1189,7 +1304,11 @@ int jot_gemm_bf16(const void* d_A, const void* d_W, const void* d_residual, void
     p.M = M; p.N = N; p.K = K; p.C = (__nv_bfloat16*)d_C; p.residual = (const __nv_bfloat16*)d_residual; p.ldc = N;
     p.status = d_status;
     if (d_scratch && (reinterpret_cast<uintptr_t>(d_scratch) & 15)) return JOT_ERR_ARG;
-    return run_gemm(di, tmA, wm, EPI_STORE, p, (cudaStream_t)stream, (float*)d_scratch, d_scratch ? scratch_bytes : 0);
+    SlabMaps tmX;
+    const bool slab = M <= kSlabMaxTokens && !d_scratch;      // with scratch: K ranges through global memory
+    if (slab) JOT_TRY(make_slab_maps(di, &tmX, d_A, M, K, K));
+    return run_gemm(di, tmA, wm, EPI_STORE, p, (cudaStream_t)stream, (float*)d_scratch, d_scratch ? scratch_bytes : 0,
+                    nullptr, slab ? &tmX : nullptr);
 }
 
 }  // extern "C"
@@ -1220,6 +1339,12 @@ int noalloc_scratch_address(float** out) {
     return JOT_OK;
 }
 }  // namespace
+
+#ifdef JOT_SLAB_TRACE
+extern "C" int jot_debug_slab_trace(unsigned long long* h_out, int n_words) {
+    return cudaMemcpyFromSymbol(h_out, g_slab_trace, (size_t)n_words * 8) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 extern "C" int jot_gemm_bf16_noalloc(const void* d_A, const void* d_W, const void* d_residual, void* d_C, int M, int N,
                                      int K, int32_t* d_status, void* stream) {
