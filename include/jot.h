@@ -149,6 +149,17 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* weights, int 
                    void* d_workspace, size_t workspace_bytes, jot_model** out);
 int jot_free_model(jot_model* m);
 
+/* The LM head gives every block of 128 active rows a CTA (256 rows a CTA pair) of its own, so one call can
+ * take at most jot_max_active_rows(number of SMs) = 128 * (SMs rounded down to even) active rows: the masked
+ * positions inside [blk_lo, blk_hi) summed over the batch, bounded by B * (blk_hi - blk_lo), which is what the
+ * entry points check (JOT_ERR_SHAPE beyond it; 18,944 on a 148-SM device).  jot_lm_head_partition reports how
+ * the head's schedule cuts `active_rows` rows and `vocab_tiles` vocabulary tiles over `n_ctas` CTAs (pair_mode:
+ * CTA pairs): row blocks and vocabulary chunks per row block.  Host arithmetic only; exported so that the
+ * schedule can be checked without a device (n_chunks >= 1 for every accepted row count). */
+int jot_max_active_rows(int n_sms);
+int jot_lm_head_partition(int active_rows, int n_ctas, int vocab_tiles, int pair_mode, int* n_row_blocks,
+                          int* n_chunks);
+
 /* Algorithm 1, "Compute logits" through "Compute confidence", for one step: the transformer forward
  * over d_tokens [B, L] (int32, read-only), then the LM head over the rows that are masked
  * (== mask_id) inside [blk_lo, blk_hi), reduced on the fly; logits are never stored.
@@ -164,6 +175,17 @@ int jot_denoise_step(jot_model* m, const int32_t* d_tokens, int B, int L, int bl
                      float* d_top1_logit, float* d_top2_logit, float* d_sumexp, int32_t* d_argmax,
                      const jot_sampling* sampling /* nullable */, int32_t* d_sampled /* [B, L], with sampling */,
                      void* stream);
+
+/* The single-step entry points (jot_denoise_step, jot_denoise_step_cached, jot_lm_head_stats) end, by default,
+ * with a 4-byte device-to-host copy of the model's status word and a synchronisation of `stream`, so that an
+ * expired device-side wait (JOT_ERR_TIMEOUT) or a token id outside [0, vocab) in d_tokens (JOT_ERR_ARG; such a
+ * row is embedded as token 0, nothing is read out of bounds) comes back as their return value.
+ * jot_set_sync(m, 0) turns that off: the calls return as soon as their kernels are enqueued, and the caller
+ * asks for the status when it wants to (jot_read_status: synchronises `stream`, returns the same codes, and
+ * clears a bad-token report so that the caller can go on with corrected input).  jot_set_sync(m, 1) restores
+ * the default.  jot_generate always reads the status itself. */
+int jot_set_sync(jot_model* m, int sync);
+int jot_read_status(jot_model* m, void* stream);
 
 /* Block-wise KV cache (Section 6.2, "Composability with KV-cache acceleration": JoT run inside a decoder that
  * caches keys and values block by block).  The paper names that decoder without defining it; the scheme
@@ -202,8 +224,9 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
  * contribute nothing), softening (Eq. 6), threshold (Eq. 7), test r >= tau in fp32 (Eq. 8).  The
  * k_transfer candidates with the largest p1 (ties to the lower position) are chosen by the transfer
  * schedule; a candidate chosen by either rule receives its argmax.  All decisions use the canvas as
- * it was on entry.  params: one struct (host) applied to all sequences; per_seq_params must be 0
- * here (per-sequence parameters are available through jot_generate).
+ * it was on entry.  params (host): one struct applied to all sequences, or, with per_seq_params != 0,
+ * B structs, one per sequence; those travel as kernel arguments, so B <= 64 then (JOT_ERR_SHAPE beyond:
+ * sequences are independent, call once per 64).
  * Outputs (device): d_n_masked [B] = candidates still masked after the update; optional
  * d_exit_reason [B, L] uint8 (bit 0 early exit, bit 1 schedule; written for finalised positions
  * only) and d_exit_step [B, L] int16 (= step_index, same positions). */
@@ -214,7 +237,7 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
                       int step_index, void* stream);
 
 /* Algorithm 1 for a batch of B independent sequences with prompts d_prompt [B, P] (int32, must not
- * contain mask_id).  Each sequence keeps its own block pointer and step counter and idles once
+ * contain mask_id; ids must lie in [0, vocab), else JOT_ERR_ARG).  Each sequence keeps its own block pointer and step counter and idles once
  * finished; the loop ends when no sequence has a masked position left, or after `steps` iterations.
  * Outputs: d_out_tokens [B, P + gen_len] (device); h_steps_used [B] (host) = denoising steps each
  * sequence actually ran (step speed-up = steps / steps_used, Section 5.1); optional

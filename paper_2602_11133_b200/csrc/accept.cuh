@@ -59,8 +59,28 @@ struct AcceptArgs {
     int32_t* n_candidates;           // [steps, B]
 };
 
+// Per-sequence parameter sets handed over as kernel arguments (the single-step entry point has no device
+// memory of its own to put them in): at most this many sequences per launch.
+constexpr int kAcceptInlineParams = 64;
+struct AcceptParamsInline {
+    AcceptParamsDev p[kAcceptInlineParams];
+};
+struct AcceptParamsNone {};
+
+template <bool INLINE> struct AcceptInlineArg { using type = AcceptParamsNone; };
+template <> struct AcceptInlineArg<true> { using type = AcceptParamsInline; };
+
+__device__ __forceinline__ AcceptParamsDev accept_pick_params(const AcceptArgs& a, const AcceptParamsInline& inl, int b) {
+    return inl.p[b];
+}
+__device__ __forceinline__ AcceptParamsDev accept_pick_params(const AcceptArgs& a, const AcceptParamsNone&, int b) {
+    return a.params ? a.params[a.per_seq_params ? b : 0] : a.uniform;
+}
+
 // Dynamic shared memory: resolved bitmap words, candidate list, candidate sum-exp, candidate flags.
-__global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const AcceptArgs a) {
+template <bool INLINE>
+__global__ void __launch_bounds__(kAcceptThreads)
+accept_freeze_kernel(const AcceptArgs a, const __grid_constant__ typename AcceptInlineArg<INLINE>::type inl) {
     extern __shared__ uint32_t sh[];
     grid_launch_dependents();
     grid_dependency_wait();
@@ -75,7 +95,7 @@ __global__ void __launch_bounds__(kAcceptThreads) accept_freeze_kernel(const Acc
     __shared__ float inv_wmax;
     __shared__ float ratio_sums[kAcceptThreads / 32], gap_sums[kAcceptThreads / 32];
 
-    const AcceptParamsDev prm = a.params ? a.params[a.per_seq_params ? b : 0] : a.uniform;
+    const AcceptParamsDev prm = accept_pick_params(a, inl, b);
     int32_t* x = a.tokens + (size_t)b * L;
 
     int lo = a.blk_lo, hi = a.blk_hi, k = a.k_transfer;

@@ -34,7 +34,10 @@ namespace jot {
 
 constexpr int kSlabThreads = 320;
 constexpr int kSlabMaxTokens = 512;        // two accumulators of 256 fp32 columns fill tensor memory
-constexpr int kSlabPreferTokens = 256;     // measured: up to here this kernel beats the token-major tiles
+#ifndef JOT_SLAB_PREFER_TOKENS
+#define JOT_SLAB_PREFER_TOKENS 256
+#endif
+constexpr int kSlabPreferTokens = JOT_SLAB_PREFER_TOKENS;   // measured: up to here this kernel beats the token-major tiles
 constexpr int kSlabMaxSmem = 226 * 1024;   // dynamic part; the static barriers take the rest of the 227 KB
 enum { SLAB_STORE = 0, SLAB_SWIGLU = 1, SLAB_QKV = 2 };
 

@@ -37,9 +37,11 @@ __device__ __forceinline__ float block_sum(float v, float* scratch /* >= 33 floa
 // The launch covers rows_per_seq consecutive canvas positions of every sequence, starting at pos0 (the whole
 // canvas: L, 0): row r is (slot, position) = (r / rows_per_seq, pos0 + r % rows_per_seq).
 // With seq_map the slots are those of a compacted batch: slot b' reads tokens[seq_map[b'], position].
+// A token id outside [0, vocab) is embedded as token 0 and reported through the status word: no read leaves E.
+constexpr int32_t kStatusBadToken = 5;
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E,
                              __nv_bfloat16* __restrict__ h, int d, int L, const int32_t* __restrict__ seq_map,
-                             int rows_per_seq, int pos0) {
+                             int rows_per_seq, int pos0, int vocab, int32_t* status) {
     grid_launch_dependents();
     grid_dependency_wait();
     const int row = blockIdx.x;
@@ -49,7 +51,12 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bflo
         b = b < 0 ? 0 : b;
     }
     const int src_row = b * L + pos0 + row % rows_per_seq;
-    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tokens[src_row] * d);
+    int tok = tokens[src_row];
+    if ((unsigned)tok >= (unsigned)vocab) {
+        if (threadIdx.x == 0 && status) atomicCAS(status, 0, kStatusBadToken);   // an expired wait, if any, stays on record
+        tok = 0;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tok * d);
     uint4* dst = reinterpret_cast<uint4*>(h + (size_t)row * d);
     for (int i = threadIdx.x; i < d / 8; i += blockDim.x) dst[i] = src[i];
 }

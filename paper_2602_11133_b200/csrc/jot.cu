@@ -380,7 +380,9 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct jot_model {
     jot_model_config cfg;
     int max_batch, max_seq;
+    DeviceInfo di_val;    // a copy: the model may outlive the thread that created it
     DeviceInfo* di;
+    bool sync_steps = true;    // single-step entry points read the status word before they return
     // borrowed weights
     const __nv_bfloat16 *embed, *lm_head, *final_norm;
     std::vector<const __nv_bfloat16*> attn_norm, mlp_norm;
@@ -595,7 +597,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
 
     {
         ProfScope ps(m, JOT_PROF_EMBED, st);
-        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d, L, seq_map, Lr, pos0);
+        launch_k(embed_kernel, dim3(M), dim3(128), 0, st, d_tokens, m->embed, m->h, d, L, seq_map, Lr, pos0, c.vocab, status);
     }
     JOT_TRY(launch_check());
     bool norm_ready = false;          // true when a fused split-K tail has already written the next norm into m->a
@@ -677,6 +679,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
                       const HeadSampling* hs = nullptr) {
     const jot_model_config& c = m->cfg;
     if (M <= 0) return JOT_OK;                       // an empty block range has no active rows
+    if (M > jot_max_active_rows(m->di->sms)) return JOT_ERR_SHAPE;   // every row block needs a CTA (pair) of its own
     GemmParams p{};
     p.M = m->R_cap; p.N = c.vocab; p.K = c.d_model; p.status = m->ctrl;
     p.d_R = m->ctrl + 1; p.rows = m->rows_out; p.bump_id = bump_id; p.bump_val = bump_val;
@@ -761,19 +764,30 @@ int check_step_args(const jot_model* m, const void* tokens, int B, int L, int bl
     return JOT_OK;
 }
 
+// Status word the kernels set: 0 ok; kStatusBadToken: a token id outside the vocabulary (the row was embedded as
+// token 0); anything else: a bounded wait expired.
+int status_code(int32_t w) { return w == 0 ? JOT_OK : (w == kStatusBadToken ? JOT_ERR_ARG : JOT_ERR_TIMEOUT); }
+
 int read_status(jot_model* m, cudaStream_t st) {
     JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 4, cudaMemcpyDeviceToHost, st));
     JOT_CUDA(cudaStreamSynchronize(st));
-    return m->h_pinned[0] ? JOT_ERR_TIMEOUT : JOT_OK;
+    const int32_t w = m->h_pinned[0];
+    if (w == kStatusBadToken) JOT_CUDA(cudaMemsetAsync(m->ctrl, 0, 4, st));     // the caller can fix its input and go on
+    return status_code(w);
 }
 
-int launch_accept(const AcceptArgs& a, cudaStream_t st) {
+int launch_accept(const AcceptArgs& a, cudaStream_t st, const AcceptParamsInline* inl = nullptr) {
     const size_t smem = accept_smem_bytes(a.L);
     if (smem > 200 * 1024) return JOT_ERR_SHAPE;
-    if (smem > 48 * 1024) {
-        JOT_CUDA(cudaFuncSetAttribute(accept_freeze_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (inl) {
+        if (smem > 48 * 1024)
+            JOT_CUDA(cudaFuncSetAttribute(accept_freeze_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        launch_k(accept_freeze_kernel<true>, dim3(a.B), dim3(kAcceptThreads), smem, st, a, *inl);
+    } else {
+        if (smem > 48 * 1024)
+            JOT_CUDA(cudaFuncSetAttribute(accept_freeze_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        launch_k(accept_freeze_kernel<false>, dim3(a.B), dim3(kAcceptThreads), smem, st, a, AcceptParamsNone{});
     }
-    launch_k(accept_freeze_kernel, dim3(a.B), dim3(kAcceptThreads), smem, st, a);
     return launch_check();
 }
 
@@ -804,6 +818,33 @@ const char* jot_status_string(int s) {
 }
 
 int jot_last_cuda_error(void) { return g_last_cuda_error; }
+
+int jot_max_active_rows(int n_sms) {
+    // more than 256 rows go through CTA pairs (256 rows per pair of SMs), so both forms allow 128 rows per SM
+    return n_sms < 2 ? 0 : 128 * (n_sms & ~1);
+}
+
+int jot_lm_head_partition(int active_rows, int n_ctas, int vocab_tiles, int pair_mode, int* n_row_blocks, int* n_chunks) {
+    if (!n_row_blocks || !n_chunks || active_rows < 0 || n_ctas <= 0 || vocab_tiles <= 0) return JOT_ERR_ARG;
+    if (pair_mode) {
+        int n_pr = 0;
+        stats_partition_pair(active_rows, n_ctas / 2, vocab_tiles, n_row_blocks, &n_pr, n_chunks);
+    } else {
+        stats_partition(active_rows, n_ctas, vocab_tiles, n_row_blocks, n_chunks);
+    }
+    return JOT_OK;
+}
+
+int jot_set_sync(jot_model* m, int sync) {
+    if (!m) return JOT_ERR_ARG;
+    m->sync_steps = sync != 0;
+    return JOT_OK;
+}
+
+int jot_read_status(jot_model* m, void* stream) {
+    if (!m) return JOT_ERR_ARG;
+    return read_status(m, (cudaStream_t)stream);
+}
 int64_t jot_launch_count(void) { return g_launches.load(); }
 
 size_t jot_workspace_bytes(const jot_model_config* cfg, int max_batch, int max_seq) {
@@ -830,7 +871,8 @@ int jot_init_model(const jot_model_config* cfg, const jot_weights* w, int max_ba
     m->cfg = *cfg;
     m->max_batch = max_batch;
     m->max_seq = max_seq;
-    m->di = di;
+    m->di_val = *di;
+    m->di = &m->di_val;
     m->embed = (const __nv_bfloat16*)w->embed;
     m->lm_head = (const __nv_bfloat16*)w->lm_head;
     m->final_norm = (const __nv_bfloat16*)w->final_norm;
@@ -937,7 +979,7 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
     }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
                               B * (blk_hi - blk_lo), st, &hs));
-    return read_status(m, st);
+    return m->sync_steps ? read_status(m, st) : JOT_OK;
 }
 
 namespace {
@@ -962,7 +1004,7 @@ int denoise_step_impl(jot_model* m, const int32_t* d_tokens, int B, int L, int b
     }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
                               B * (blk_hi - blk_lo), st, &hs));
-    return read_status(m, st);
+    return m->sync_steps ? read_status(m, st) : JOT_OK;
 }
 }  // namespace
 
@@ -1020,19 +1062,24 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
                       int16_t* d_exit_step, int step_index, void* stream) {
     if (!params || !d_tokens || !d_top1 || !d_top2 || !d_sumexp || !d_argmax) return JOT_ERR_ARG;
     if (B <= 0 || L <= 0 || blk_lo < 0 || blk_hi > L || blk_lo > blk_hi || k_transfer < 0) return JOT_ERR_ARG;
-    if (per_seq_params) return JOT_ERR_ARG;   // per-sequence parameters are available through jot_generate
-    if (!params_ok(params)) return JOT_ERR_ARG;
+    const int n_par = per_seq_params ? B : 1;
+    if (n_par > kAcceptInlineParams) return JOT_ERR_SHAPE;       // B parameter sets travel as kernel arguments
+    for (int i = 0; i < n_par; ++i)
+        if (!params_ok(params + i)) return JOT_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
+    static_assert(sizeof(AcceptParamsDev) == sizeof(jot_params), "parameter struct layouts must agree");
     AcceptArgs a{};
-    a.uniform = AcceptParamsDev{params->tau_max, params->tau_min, params->gamma, params->D, params->eps,
-                                params->schedule_after_exit, params->gate, params->prob_threshold, params->gap_threshold};
+    AcceptParamsInline inl{};
+    memcpy(inl.p, params, (size_t)n_par * sizeof(jot_params));
+    a.uniform = inl.p[0];
     a.params = nullptr;
+    a.per_seq_params = per_seq_params ? 1 : 0;
     a.mask_id = mask_id; a.tokens = d_tokens; a.B = B; a.L = L;
     a.blk_lo = blk_lo; a.blk_hi = blk_hi; a.k_transfer = k_transfer;
     a.top1 = d_top1; a.top2 = d_top2; a.sumexp = d_sumexp; a.argmax = d_argmax;
     a.n_masked = d_n_masked; a.exit_reason = d_exit_reason; a.exit_step = d_exit_step; a.step_index = step_index;
     a.state = nullptr;
-    JOT_TRY(launch_accept(a, st));
+    JOT_TRY(launch_accept(a, st, per_seq_params ? &inl : nullptr));
     return JOT_OK;
 }
 
@@ -1075,7 +1122,10 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
     auto outcome = [&](int slot, bool* finished) -> int {      // wait for a step's control words
         JOT_CUDA(cudaEventSynchronize(m->step_done[slot]));
         const int32_t* w = m->h_pinned + 4 * slot;
-        if (w[0]) return JOT_ERR_TIMEOUT;
+        if (w[0]) {
+            if (w[0] == kStatusBadToken) cudaMemsetAsync(m->ctrl, 0, 4, st);
+            return status_code(w[0]);
+        }
         *finished = w[2] == 0;
         if (!*finished) B_act = w[2];
         return JOT_OK;
@@ -1134,7 +1184,11 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
                 }
                 JOT_CUDA(cudaMemcpyAsync(m->h_pinned, m->ctrl, 16, cudaMemcpyDeviceToHost, st));
                 JOT_CUDA(cudaStreamSynchronize(st));
-                if (m->h_pinned[0]) return JOT_ERR_TIMEOUT;
+                if (m->h_pinned[0]) {
+                    const int32_t w0 = m->h_pinned[0];
+                    if (w0 == kStatusBadToken) cudaMemsetAsync(m->ctrl, 0, 4, st);
+                    return status_code(w0);
+                }
                 ++n_passes;
                 if (m->h_pinned[2] == 0) break;              // no sequence has a masked position left in this block
             }

@@ -21,6 +21,7 @@ EXPORTS = [
     "jot_denoise_step", "jot_lm_head_stats", "jot_accept_freeze", "jot_generate", "jot_gemm_bf16",
     "jot_launch_count", "jot_profile", "jot_profile_read", "jot_gemm_bf16_noalloc",
     "jot_selftest_wait_expiry", "jot_kv_cache_bytes", "jot_attach_kv_cache", "jot_denoise_step_cached",
+    "jot_max_active_rows", "jot_lm_head_partition", "jot_set_sync", "jot_read_status",
 ]
 
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -129,6 +130,10 @@ def _lib():
                                               C.c_void_p, C.c_void_p]
         lib.jot_launch_count.restype = C.c_int64
         lib.jot_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        lib.jot_max_active_rows.argtypes = [C.c_int]
+        lib.jot_lm_head_partition.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        lib.jot_set_sync.argtypes = [C.c_void_p, C.c_int]
+        lib.jot_read_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.jot_profile.argtypes = [C.c_void_p, C.c_int]
         lib.jot_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int]
         _LIB = lib
@@ -159,6 +164,18 @@ def _sampling_args(sampling, out, B, L, device):
     if out.sampled is None:
         out.sampled = torch.zeros(B, L, dtype=torch.int32, device=device)
     return C.byref(sampling), _ptr(out.sampled, torch.int32, "sampled")
+
+
+def max_active_rows(n_sms: int) -> int:
+    return int(_lib().jot_max_active_rows(n_sms))
+
+
+def lm_head_partition(active_rows: int, n_ctas: int, vocab_tiles: int, pair_mode: bool):
+    """(row blocks, vocabulary chunks per row block) of the LM-head schedule; host arithmetic only."""
+    n_rb, n_ch = C.c_int(0), C.c_int(0)
+    _check(_lib().jot_lm_head_partition(active_rows, n_ctas, vocab_tiles, int(pair_mode), C.byref(n_rb), C.byref(n_ch)),
+           "jot_lm_head_partition")
+    return n_rb.value, n_ch.value
 
 
 def launch_count() -> int:
@@ -253,6 +270,14 @@ class Model:
         except Exception:
             pass
 
+    def set_sync(self, sync: bool) -> None:
+        """sync=False: the single-step calls return once their kernels are enqueued; read_status() asks later."""
+        _check(_lib().jot_set_sync(self.handle, int(sync)), "jot_set_sync")
+
+    def read_status(self) -> None:
+        """Synchronise the current stream and raise if a kernel reported a failure since the last read."""
+        _check(_lib().jot_read_status(self.handle, _stream()), "jot_read_status")
+
     def profile(self, enable: bool) -> None:
         """Start (and clear) or stop per-kernel-class event timing."""
         _check(_lib().jot_profile(self.handle, int(enable)), "jot_profile")
@@ -335,12 +360,20 @@ class Model:
         return out, list(used), int(passes.value)
 
 
-def accept_freeze(params: Params, mask_id: int, tokens: torch.Tensor, blk_lo: int, blk_hi: int, k_transfer: int,
+def accept_freeze(params, mask_id: int, tokens: torch.Tensor, blk_lo: int, blk_hi: int, k_transfer: int,
                   stats: Stats, n_masked: Optional[torch.Tensor] = None, exit_reason: Optional[torch.Tensor] = None,
                   exit_step: Optional[torch.Tensor] = None, step_index: int = 0) -> None:
-    """In-place acceptance / freeze update of tokens [B, L] (Section 4.1, Algorithm 1)."""
+    """In-place acceptance / freeze update of tokens [B, L] (Section 4.1, Algorithm 1).
+    params: one Params for the whole batch, or a list of B (one per sequence)."""
     B, L = tokens.shape
-    _check(_lib().jot_accept_freeze(C.byref(params), 0, mask_id, _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo,
+    per_seq = isinstance(params, (list, tuple))
+    if per_seq:
+        if len(params) != B:
+            raise ValueError("need one Params per sequence")
+        parr = (Params * B)(*params)
+    else:
+        parr = (Params * 1)(params)
+    _check(_lib().jot_accept_freeze(parr, int(per_seq), mask_id, _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo,
                                     blk_hi, k_transfer, _ptr(stats.top1, torch.float32, "top1"),
                                     _ptr(stats.top2, torch.float32, "top2"), _ptr(stats.sumexp, torch.float32, "sumexp"),
                                     _ptr(stats.argmax, torch.int32, "argmax"), _ptr(n_masked, torch.int32, "n_masked"),

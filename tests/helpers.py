@@ -17,6 +17,7 @@ from oracle import model_oracle as mo
 
 REL_TOL = 2e-2
 GAP_TOL = 1e-3
+LAST_COMPARE = {}        # counts of the latest compare_stats call (rows, inside_margin, inside_strict_margin, argmax_differs)
 
 
 def oracle_stats_for_rows(logits_rows: torch.Tensor, mask_id) -> List[jo.RowStats]:
@@ -32,7 +33,7 @@ def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowS
     tolerance itself implies: two logits that may each move by rel*scale can swap when their gap is below
     2*rel*scale.  Exempt rows are counted, and their argmax must still be the oracle's runner-up region:
     the GPU's top-1 logit has to be within tolerance of the oracle's."""
-    near = 0
+    near = strict = differ = 0
     for r, st in enumerate(want):
         scale = max(abs(st.m1), abs(st.m2), 1.0)
         gap_tol = max(GAP_TOL, 2 * rel * scale) if gap_from_tolerance else GAP_TOL
@@ -42,8 +43,14 @@ def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowS
         assert abs(math.log(got_sumexp[r]) - math.log(st.S)) <= rel * scale, (r, got_sumexp[r], st.S)
         if st.m1 - st.m2 < gap_tol:
             near += 1                     # top-2 gap inside the margin: either index is a valid argmax
+            strict += int(st.m1 - st.m2 < GAP_TOL)
+            differ += int(int(got_argmax[r]) != st.i1)
         else:
             assert int(got_argmax[r]) == st.i1, (r, int(got_argmax[r]), st.i1, st.m1 - st.m2)
+    LAST_COMPARE.update(rows=len(want), inside_margin=near, inside_strict_margin=strict, argmax_differs=differ)
+    if gap_from_tolerance:
+        print(f"compare_stats: {len(want)} rows; top-2 gap inside the widened margin: {near} "
+              f"(of which inside the strict {GAP_TOL:g} margin: {strict}); argmax actually different: {differ}")
     return len(want), near
 
 
@@ -117,3 +124,51 @@ def replay_trajectory(jot, model, tr: jo.Trajectory, params: jo.JotParams, mask_
             assert near_tau or near_gap or near_rank, (n, i, got[i], want[i], rep.ratio.get(i), rep.tau.get(i))
             excused += 1
     return len(tr.canvases), excused
+
+
+def manual_generate(jot, model, prompt_row, G, T, jp, block_len, mask_id, bump=None, sampling=None):
+    """Algorithm 1 for ONE sequence driven from the host through the single-step entry points (jot_denoise_step +
+    jot_accept_freeze), free-running on the GPU's own canvas.  jot_generate must give the very same tokens and
+    step count: both run the same kernels on the same state, so this comparison needs no tolerance and no
+    condition.  sampling = (temperature, seed).  Returns (tokens list, steps_used)."""
+    import torch
+    P = len(prompt_row)
+    Lb = block_len or G
+    nb = G // Lb
+    Tb = T // nb
+    ks = jo.transfer_counts(Lb, Tb)
+    x = torch.tensor([list(prompt_row) + [mask_id] * G], dtype=torch.int32, device="cuda")
+    d_bump = dict(bump_id=bump[0].cuda(), bump_val=bump[1].cuda()) if bump is not None else {}
+    n_masked = torch.zeros(1, dtype=torch.int32, device="cuda")
+    used = 0
+    for blk in range(nb):
+        lo, hi = P + blk * Lb, P + (blk + 1) * Lb
+        for s in range(Tb):
+            if int((x[0, lo:hi] == mask_id).sum()) == 0:
+                break
+            if sampling is not None:
+                st = model.denoise_step(x, lo, hi, sampling=jot.Sampling(sampling[0], sampling[1], used), **d_bump)
+                st = jot.Stats(st.top1, st.top2, st.sumexp, st.sampled)
+            else:
+                st = model.denoise_step(x, lo, hi, **d_bump)
+            jot.accept_freeze(jp, mask_id, x, lo, hi, ks[s], st, n_masked)
+            used += 1
+    return x.cpu()[0].tolist(), used
+
+
+def assert_generate_matches(jot, model, prompt, G, T, jp, block_len, mask_id, bump, out, used, tr, excused, label="",
+                            sampling=None):
+    """What is asserted about a free-running jot_generate result, unconditionally and conditionally:
+    always   the library's loop equals the host-driven loop over the single-step entry points, token for token;
+    if the teacher-forced replay excused nothing, also the oracle's trajectory, token for token and step for step;
+    otherwise the branch taken is printed (a decision inside the margin makes the two runs different samples)."""
+    got = out.cpu()[0].tolist()
+    man, man_used = manual_generate(jot, model, prompt[0].tolist(), G, T, jp, block_len, mask_id, bump, sampling)
+    assert got == man and used[0] == man_used, "jot_generate differs from the host-driven loop"
+    if excused == 0:
+        assert used[0] == tr.steps_used and got == tr.x
+        print(f"{label}free-running run equals the oracle ({tr.steps_used} steps)")
+    else:
+        same = sum(int(a == b) for a, b in zip(got, tr.x))
+        print(f"{label}free-running equality with the oracle NOT asserted ({excused} excused decisions in the replay); "
+              f"{same}/{len(got)} tokens equal, {used[0]} vs {tr.steps_used} steps")

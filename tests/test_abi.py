@@ -43,3 +43,42 @@ def test_host_side_calls_without_device_work():
     # argument errors are reported before anything touches a device
     assert lib.jot_generate(None, None, 0, None, None, 1, 1, None, None, None, None, None, None) == -1
     assert lib.jot_accept_freeze(None, 0, 0, None, 1, 1, 0, 1, 1, None, None, None, None, None, None, None, 0, None) == -1
+
+
+def test_lm_head_schedule_gives_every_accepted_row_count_a_chunk():
+    """The LM head's split of (row blocks) x (vocabulary chunks) over the CTAs, on the host: every active-row
+    count the entry points accept must get at least one vocabulary chunk per row block (zero chunks would leave
+    rows without statistics), and the chunks must cover all vocabulary tiles."""
+    from paper_2602_11133_b200 import jot
+    for sms in (148, 132, 8, 3):
+        limit = jot.max_active_rows(sms)
+        assert limit == 128 * (sms - sms % 2)
+        grid = min(sms, 256)
+        for vocab in (4096, 126464, 152064):
+            rows = sorted(set(list(range(1, 300)) + list(range(300, limit, 997)) + [limit - 1, limit]))
+            for R in rows:
+                if R > limit:
+                    continue
+                # the same choice of kernel shape as the library: 128-wide tiles up to 128 rows, 256-wide up to
+                # 256 rows, CTA pairs beyond
+                pair = R > 256
+                bn = 128 if R <= 128 else 256
+                n_vt = (vocab + bn - 1) // bn
+                n_rb, n_ch = jot.lm_head_partition(R, grid & ~1 if pair else grid, n_vt, pair)
+                assert n_rb == (R + 127) // 128
+                assert 1 <= n_ch <= n_vt, (sms, vocab, R, n_rb, n_ch)
+                units = (n_rb + 1) // 2 if pair else n_rb
+                assert units * n_ch <= (grid // 2 if pair else grid)
+        n_rb, n_ch = jot.lm_head_partition(limit + 128, grid & ~1, 988, True)
+        assert n_ch == 0              # beyond the limit the schedule has no room: that is why the entry points refuse it
+
+
+def test_new_host_side_argument_checks():
+    lib = ctypes.CDLL(jot_build.build())
+    from paper_2602_11133_b200 import jot
+    assert lib.jot_set_sync(None, 0) == -1 and lib.jot_read_status(None, None) == -1
+    assert lib.jot_lm_head_partition(10, 148, 988, 0, None, None) == -1
+    # per-sequence parameter sets travel as kernel arguments: at most 64 sequences per call
+    pars = (jot.Params * 65)(*[jot.Params() for _ in range(65)])
+    one = ctypes.c_void_p(16)        # never dereferenced: the size check comes first
+    assert lib.jot_accept_freeze(pars, 1, 0, one, 65, 8, 0, 8, 1, one, one, one, one, None, None, None, 0, None) == -2

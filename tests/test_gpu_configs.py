@@ -4,6 +4,7 @@ with the planted bump (batch > 1, per-sequence block pointers)."""
 import pytest
 import torch
 
+import helpers
 from helpers import GAP_TOL, REL_TOL, compare_stats, oracle_stats_for_rows, replay_trajectory
 from oracle import jot_oracle as jo
 from oracle import model_oracle as mo
@@ -66,7 +67,7 @@ def test_llada_long_generation_shape_step_two_layers(jot):
     torch.cuda.synchronize()
     w_cpu = inputs.weights_to(w_gpu, "cpu")
     tok = tokens.cpu()
-    n_near = 0
+    n_near = n_differ = 0
     for b in (0, 7, B - 1):
         h = mo.hidden_states(g, w_cpu, tok[b:b + 1])
         sel = list(range(P, P + Lb, 3))                                    # 11 of the block's 32 rows
@@ -79,9 +80,15 @@ def test_llada_long_generation_shape_step_two_layers(jot):
         # tolerance, and two logits closer than twice that may swap places (counted)
         n, near = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), want, rel=REL_TOL / 2,
                                 gap_from_tolerance=True)
-        assert n == len(sel) and near <= 4
+        assert n == len(sel)
         n_near += near
-    print(f"{n_near} of 33 sampled rows had a top-2 gap inside the margin")
+        n_differ += helpers.LAST_COMPARE["argmax_differs"]
+    # What the arithmetic predicts: the margin is 2 * 0.01 * 5.6 = 0.11 logits; where the planted bump loses (about
+    # half of the rows) the two largest of 126k Gaussian logits (sigma 1.28) lie ~0.26 apart on average, so about
+    # 0.5 * (1 - exp(-0.11 / 0.26)) = 17 % of the rows, 5-6 of 33, fall inside it.  Inside the margin the argmax only
+    # flips when the noise (~0.02) exceeds the actual gap: a fifth of those.  Caps at twice the prediction.
+    print(f"{n_near} of 33 sampled rows had a top-2 gap inside the margin; argmax actually differed on {n_differ}")
+    assert n_near <= 11 and n_differ <= 3
     model.close()
 
 

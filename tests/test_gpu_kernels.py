@@ -148,6 +148,74 @@ def test_accept_freeze_matches_oracle(jot, B, L, P, lo, hi, k, params):
     assert torch.equal(got[keep], torch.from_numpy(tokens)[keep])
 
 
+# the hyper-parameter sweep of the paper's Dream runs (Appendix, "Hyperparameter sweep" table): tau_max x (gamma, D)
+SWEEP = [jo.JotParams(float(t), 1.0, g, D) for t in (60, 90, 120) for g, D in ((0.3, 8), (0.5, 8), (0.5, 16), (0.7, 8))]
+
+
+@pytest.mark.parametrize("B,L,P,lo,hi,k", [(8, 512, 256, 256, 512, 1), (3, 704, 192, 224, 256, 1)])
+@pytest.mark.parametrize("params", SWEEP, ids=lambda p: f"tau{p.tau_max:g}-g{p.gamma:g}-D{p.D}")
+def test_accept_freeze_sweep_settings(jot, B, L, P, lo, hi, k, params):
+    """Every one of the 12 sweep settings, on the Dream-shaped canvas (batch 8, 256 + 256) and on a block of a
+    long canvas: canvas, masked count and exit reasons equal to the oracle's outside its near-margin list."""
+    V, mask_id = 152064, 151666
+    tokens, top1, top2, sumexp, argmax = random_accept_case(77 * B + params.D, B, L, P, mask_id, V)
+    want, reps = oracle_accept_batch(torch.from_numpy(tokens), top1, top2, sumexp, argmax, params, mask_id, lo, hi, k)
+    d_tok = torch.from_numpy(tokens).cuda()
+    st = jot.Stats(*[torch.from_numpy(t).cuda() for t in (top1, top2, sumexp, argmax)])
+    n_masked = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    reason = torch.zeros(B, L, dtype=torch.uint8, device="cuda")
+    jot.accept_freeze(jot.Params(params.tau_max, params.tau_min, params.gamma, params.D, params.eps), mask_id, d_tok,
+                      lo, hi, k, st, n_masked, reason)
+    got, reason = d_tok.cpu(), reason.cpu().numpy()
+    n_exit = 0
+    for b in range(B):
+        nm = set(reps[b].near_margin)
+        assert len(nm) <= 2
+        for i in range(L):
+            if i not in nm:
+                assert int(got[b, i]) == int(want[b, i]), (b, i, reps[b].ratio.get(i), reps[b].tau.get(i))
+        if not nm:
+            assert int(n_masked[b]) == int((want[b, lo:hi] == mask_id).sum())
+            assert sorted(np.nonzero(reason[b] & 1)[0].tolist()) == sorted(reps[b].exited)
+            assert sorted(np.nonzero(reason[b] & 2)[0].tolist()) == sorted(reps[b].scheduled)
+        n_exit += len(reps[b].exited)
+    assert n_exit > 0                      # the setting decides something on this input
+
+
+def test_accept_freeze_per_sequence_parameters(jot):
+    """One call, a different parameter set for every sequence: each sequence must come out as the oracle run
+    with ITS set, and at least two sequences must differ from what a shared set would have given them."""
+    V, mask_id, B, L, P = 5000, 4321, 6, 384, 128
+    tokens, top1, top2, sumexp, argmax = random_accept_case(4242, B, L, P, mask_id, V)
+    sets = [jo.DREAM_DEFAULT, jo.LLADA_DEFAULT, jo.JotParams(60, 1, 0.7, 8), jo.JotParams(120, 1, 0.3, 32),
+            jo.JotParams(5, 5, 0.5, 8), jo.JotParams(90, 30, 0.9, 16)]
+    d_tok = torch.from_numpy(tokens).cuda()
+    st = jot.Stats(*[torch.from_numpy(t).cuda() for t in (top1, top2, sumexp, argmax)])
+    n_masked = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    jot.accept_freeze([jot.Params(p.tau_max, p.tau_min, p.gamma, p.D, p.eps) for p in sets], mask_id, d_tok, P, L, 2,
+                      st, n_masked)
+    got = d_tok.cpu()
+    differs_from_shared = 0
+    for b, prm in enumerate(sets):
+        sl = slice(b, b + 1)
+        want, reps = oracle_accept_batch(torch.from_numpy(tokens[sl]), top1[sl], top2[sl], sumexp[sl], argmax[sl], prm,
+                                         mask_id, P, L, 2)
+        nm = set(reps[0].near_margin)
+        assert len(nm) <= 2
+        for i in range(L):
+            if i not in nm:
+                assert int(got[b, i]) == int(want[0, i]), (b, i)
+        shared, _ = oracle_accept_batch(torch.from_numpy(tokens[sl]), top1[sl], top2[sl], sumexp[sl], argmax[sl], sets[0],
+                                        mask_id, P, L, 2)
+        differs_from_shared += int(not torch.equal(shared, want))
+    assert differs_from_shared >= 2
+    with pytest.raises(jot.JotError) as e:       # more sequences than parameter sets fit into one launch
+        big = torch.from_numpy(np.repeat(tokens[:1], 65, axis=0).copy()).cuda()
+        st65 = jot.Stats(*[torch.from_numpy(np.repeat(t[:1], 65, axis=0).copy()).cuda() for t in (top1, top2, sumexp, argmax)])
+        jot.accept_freeze([jot.Params()] * 65, mask_id, big, P, L, 1, st65)
+    assert e.value.status == -2
+
+
 def test_accept_freeze_degenerate_cases(jot):
     V, mask_id, B, L = 100, 99, 2, 64
     tokens, top1, top2, sumexp, argmax = random_accept_case(5, B, L, 8, mask_id, V)

@@ -5,7 +5,8 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import GAP_TOL, REL_TOL, compare_stats, oracle_stats_for_rows, replay_trajectory
+from helpers import (GAP_TOL, REL_TOL, assert_generate_matches, compare_stats, oracle_stats_for_rows,
+                     replay_trajectory)
 from oracle import jot_oracle as jo
 from oracle import model_oracle as mo
 from paper_2602_11133_b200 import inputs
@@ -97,13 +98,14 @@ def test_tiny_generation_teacher_forced_and_free_running(jot, params, block_len,
     if bumped:
         assert excused <= 2
         assert tr.steps_used < T          # the bump makes positions exit early
+    else:
+        assert excused <= 0.75 * len(tr.canvases)      # measured: 38-40 of 63 picks among near-equal confidences
 
     out, used, passes = model.generate(prompt.cuda(), G, T, jp, block_len, **d_bump)
     got = out.cpu()[0].tolist()
     assert got[:P] == prompt[0].tolist() and all(t != g.mask_id for t in got)
     assert 1 <= used[0] <= T and passes == used[0]
-    if excused == 0:
-        assert used[0] == tr.steps_used and got == tr.x
+    assert_generate_matches(jot, model, prompt, G, T, jp, block_len, g.mask_id, bump, out, used, tr, excused)
     model.close()
 
 
@@ -182,6 +184,54 @@ def test_argument_validation(jot):
     model.close()
 
 
+def test_token_id_outside_the_vocabulary_is_reported_not_read(jot):
+    """A token id outside [0, vocab) must come back as an argument error: the row is embedded as token 0 (no read
+    leaves the embedding matrix), the status word records it, and the model works again on corrected input."""
+    g = inputs.TINY
+    w_gpu = inputs.weights_to(inputs.model_weights(g, seed=0, n_layers=1), "cuda")
+    model = jot.Model(g, w_gpu, 2, 64)
+    good = inputs.partially_masked_canvas(3, 2, 16, 48, g.vocab, g.mask_id, 0.5).cuda()
+    ref = model.denoise_step(good, 16, 64)
+    for bad_id in (g.vocab, g.vocab + 12345, -1, -2 ** 31):
+        bad = good.clone()
+        bad[1, 3] = bad_id
+        with pytest.raises(jot.JotError) as e:
+            model.denoise_step(bad, 16, 64)
+        assert e.value.status == -1
+        again = model.denoise_step(good, 16, 64)                   # the report was cleared; same result as before
+        assert torch.equal(again.top1, ref.top1) and torch.equal(again.argmax, ref.argmax)
+    with pytest.raises(jot.JotError) as e:                         # the generate loop reports it the same way
+        model.generate(torch.full((1, 8), g.vocab, dtype=torch.int32, device="cuda"), 8, 8, jot.Params())
+    assert e.value.status == -1
+    out, used, _ = model.generate(good[:1, :16].contiguous(), 16, 16, jot.Params())
+    assert (out != g.mask_id).all()
+    model.close()
+
+
+def test_steps_without_a_synchronisation_per_call(jot):
+    """jot_set_sync(0): the single-step calls only enqueue; the status is read when the caller asks.  Results are
+    those of the synchronous calls, and a failure that happened in between is still reported by jot_read_status."""
+    g = inputs.TINY
+    w_gpu = inputs.weights_to(inputs.model_weights(g, seed=0), "cuda")
+    model = jot.Model(g, w_gpu, 1, 96)
+    x = inputs.partially_masked_canvas(4, 1, 32, 64, g.vocab, g.mask_id, 0.6).cuda()
+    ref = model.denoise_step(x, 32, 96)
+    model.set_sync(False)
+    outs = [model.denoise_step(x, 32, 96) for _ in range(5)]       # five steps in flight, no host round trip
+    model.read_status()
+    for o in outs:
+        assert torch.equal(o.top1, ref.top1) and torch.equal(o.sumexp, ref.sumexp) and torch.equal(o.argmax, ref.argmax)
+    bad = x.clone()
+    bad[0, 0] = g.vocab
+    model.denoise_step(bad, 32, 96)                                # returns ok: nothing has been read yet
+    with pytest.raises(jot.JotError) as e:
+        model.read_status()
+    assert e.value.status == -1
+    model.read_status()                                            # cleared
+    model.set_sync(True)
+    model.close()
+
+
 # ---------------------------------------------------------------- sampling-based finalisation (Section 4.1)
 def sampled_oracle_trajectory(g, w_cpu, prompt_row, G, T, params, block_len, bump, temperature, seed, seq_index=0,
                               bump_row=0):
@@ -253,8 +303,8 @@ def test_tiny_generation_with_sampled_finalisation(jot, params, block_len, tempe
     out, used, passes = model.generate(prompt.cuda(), G, T, jp, block_len, temperature=temperature, seed=seed, **d_bump)
     got = out.cpu()[0].tolist()
     assert got[:P] == prompt[0].tolist() and all(t != g.mask_id for t in got) and passes == used[0]
-    if excused == 0:
-        assert used[0] == tr.steps_used and got == tr.x
+    assert_generate_matches(jot, model, prompt, G, T, jp, block_len, g.mask_id, bump, out, used, tr, excused,
+                            label="sampled: ", sampling=(temperature, seed))
     # temperature 0 is the argmax path whatever the seed
     o0, u0, _ = model.generate(prompt.cuda(), G, T, jp, block_len, temperature=0.0, seed=seed, **d_bump)
     o1, u1, _ = model.generate(prompt.cuda(), G, T, jp, block_len, **d_bump)
@@ -330,8 +380,9 @@ def test_generation_trace_matches_oracle(jot):
     assert all(1 <= e <= used[0] and r in (1, 2, 3) for e, r in zip(es[P:], er[P:]))
     assert all(n == 0 and m == 0.0 for n, m in zip(nc[used[0]:], mr[used[0]:])) and all(n > 0 for n in nc[:used[0]])
     assert sum(1 for r in er[P:] if r & 2) >= used[0] - (G // block_len)      # the schedule reveals one per step
+    assert_generate_matches(jot, model, prompt, G, T, jp, block_len, g.mask_id, bump, out, used, tr, excused,
+                            label="trace: ")
     if excused == 0:
-        assert used[0] == tr.steps_used and out.cpu()[0].tolist() == tr.x
         assert es == tr.exit_step
         want_reason = [0] * L
         for rep in tr.reports:
@@ -389,8 +440,15 @@ def test_generation_under_the_global_early_commit_gate(jot):
     # (2-layer model: the measured logit error is ~2e-3, so 0.02 on a mean of gaps is a wide berth)
     margins = [abs(float(np.mean(gaps)) - thr) for gaps in step_gaps(tr, g, w_cpu, bump)]
     print(f"threshold {thr}: oracle used {tr.steps_used} steps, smallest |mean gap - threshold| {min(margins):.3f}")
+    from helpers import manual_generate
+    jp_gap = jot.Params(gate=jot.GATE_GLOBAL_GAP, gap_threshold=thr)
+    man, man_used = manual_generate(jot, model, prompt[0].tolist(), G, T, jp_gap, Lb, g.mask_id, bump)
+    assert out.cpu()[0].tolist() == man and used[0] == man_used        # always: library loop == host-driven loop
     if min(margins) >= 0.02:
         assert used[0] == tr.steps_used and out.cpu()[0].tolist() == tr.x
+        print("free-running run equals the oracle")
+    else:
+        print("free-running equality with the oracle NOT asserted: a step's mean gap sits within 0.02 of the threshold")
     model.close()
 
 

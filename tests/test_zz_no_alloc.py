@@ -8,6 +8,7 @@ collected last on purpose, so a failure here cannot hide the result of any other
 import pytest
 import torch
 
+from helpers import bf16_matmul_oracle
 from paper_2602_11133_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -42,6 +43,9 @@ def test_noalloc_projection_matches_ordinary_entry_point_twice(jot):
         tol = 2.0 ** -8 * ref.abs() + 1e-3 * ref.abs().max()
         assert ((got - ref).abs() <= tol).all()
         assert ref.abs().max().item() > 0.1
+        # ... and against the float64 definition of the projection, with the same tolerance
+        exact = bf16_matmul_oracle(a.cpu(), w.cpu(), None if res is None else res.cpu())
+        assert ((got.double() - exact).abs() <= 2.0 ** -8 * exact.abs() + 1e-3 * exact.abs().max()).all()
 
 
 def test_noalloc_projection_rejects_what_does_not_fit(jot):
