@@ -12,6 +12,14 @@ import torch.multiprocessing as mp
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+def free_port():
+    """A TCP port nobody listens on right now (two test runs on one host must not meet on a fixed number)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def _rank_main(rank, world, port, out_dir):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     sys.path.insert(0, ROOT)
@@ -28,7 +36,7 @@ def _rank_main(rank, world, port, out_dir):
 
 
 def test_two_gloo_ranks_agree_on_max_time_and_aggregate(tmp_path):
-    world, port = 2, 29613
+    world, port = 2, free_port()
     mp.spawn(_rank_main, args=(world, port, str(tmp_path)), nprocs=world, join=True)
     res = [json.load(open(tmp_path / f"r{r}.json")) for r in range(world)]
     for r in res:
@@ -37,7 +45,7 @@ def test_two_gloo_ranks_agree_on_max_time_and_aggregate(tmp_path):
 
 
 def test_reference_arm_runs_on_rank_zero_only():
-    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1", MASTER_ADDR="127.0.0.1", MASTER_PORT="29614")
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(free_port()))
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
                         "--gpus", "2"], env=env, capture_output=True, text=True, timeout=300)
     assert p.returncode == 0 and p.stdout.strip() == ""
