@@ -19,7 +19,9 @@ choice is visible at the call site):
   * the window sum of Eq. 5 skips j = i (i is masked) and positions outside the
     canvas contribute nothing; w_max is not adjusted at the canvas edges;
   * the transfer schedule is "k highest max-probability positions", with k from
-    a fixed per-block table, and it ranks ALL currently masked candidates; its
+    a fixed per-block table (or, as an option, the share of what is still
+    masked that keeps the block on pace: fractional_transfer_count), and it
+    ranks ALL currently masked candidates; its
     mask is OR-ed with the early-exit mask (Section 4.2 "Implementation
     details"); `schedule_after_exit=True` gives the other reading of
     Algorithm 1 (schedule ranks only what early exit left masked);
@@ -215,6 +217,18 @@ def transfer_counts(block_len: int, steps_per_block: int) -> List[int]:
     return [base + (1 if s < rem else 0) for s in range(steps_per_block)]
 
 
+def fractional_transfer_count(n_masked: int, steps_left: int) -> int:
+    """The adaptive alternative to the fixed table: with `steps_left` steps of the block still to run (this one
+    included), reveal the share of what is STILL masked that keeps the block on pace to end with its last step:
+    ceil(n_masked / steps_left).  The paper leaves the schedule to "the model's default unmasking schedule"
+    (Section 4.2, "Interaction with transfer schedules"); samplers of the Dream family reveal a fraction of the
+    remaining masked positions per step, which is this rule up to how the fraction is rounded.  Rounding up is this
+    build's reading: it reveals at least one position while any is masked (every step makes progress, the block
+    ends within its steps), and without early exits it reproduces transfer_counts exactly."""
+    assert steps_left >= 1
+    return -(-n_masked // steps_left)
+
+
 # ----------------------------------------------------------------------------
 # one acceptance / freeze update (inner part of Algorithm 1)
 # ----------------------------------------------------------------------------
@@ -287,7 +301,8 @@ def generate(logits_fn: Callable[[List[int], List[int]], dict], prompt: Sequence
              steps: int, p: JotParams, mask_id: int, block_len: Optional[int] = None,
              exclude_mask_token: bool = True, schedule_after_exit: bool = False,
              stats_fn: Optional[Callable[[List[int], List[int]], dict]] = None,
-             sampling: Optional[Tuple[float, int]] = None, seq_index: int = 0) -> Trajectory:
+             sampling: Optional[Tuple[float, int]] = None, seq_index: int = 0,
+             schedule: str = "fixed") -> Trajectory:
     """Algorithm 1 for one sequence.
 
     logits_fn(x, rows) returns {i: logits row (length K)} for the requested masked positions;
@@ -295,7 +310,10 @@ def generate(logits_fn: Callable[[List[int], List[int]], dict], prompt: Sequence
     sampling = (temperature, seed): finalised positions receive a sample from softmax(l / temperature) drawn
     with sample_tokens_fast, keyed by the 0-based index of the forward pass and the position's flat canvas
     index seq_index * L + i; the acceptance decisions themselves do not change.
+    schedule = "fixed": the per-block table of transfer_counts; "fractional": fractional_transfer_count of what
+    is still masked in the block and the steps the block has left.
     """
+    assert schedule in ("fixed", "fractional")
     P = len(prompt)
     Lb = gen_len if block_len is None else block_len
     assert gen_len % Lb == 0
@@ -322,7 +340,8 @@ def generate(logits_fn: Callable[[List[int], List[int]], dict], prompt: Sequence
                                                    sampling[1], traj.steps_used, seq_index * len(x) + i)[0] for i in A}
             traj.canvases.append(list(x))
             traj.blocks.append((lo, hi))
-            rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[s], schedule_after_exit, drawn)
+            k = ks[s] if schedule == "fixed" else fractional_transfer_count(len(A), Tb - s)
+            rep = accept_freeze(x, stats, p, mask_id, lo, hi, k, schedule_after_exit, drawn)
             traj.reports.append(rep)
             traj.steps_used += 1
             for i in set(rep.exited) | set(rep.scheduled):

@@ -313,6 +313,54 @@ def test_generate_schedule_table_restarts_in_every_block():
     assert [cv.count(M) for cv in tr.canvases] == [12, 10, 8, 7, 6, 4, 2, 1]
 
 
+def test_fractional_schedule_counts():
+    # hand-worked: ceil(remaining / steps left)
+    assert jo.fractional_transfer_count(6, 4) == 2 and jo.fractional_transfer_count(4, 3) == 2
+    assert jo.fractional_transfer_count(2, 2) == 1 and jo.fractional_transfer_count(1, 1) == 1
+    assert jo.fractional_transfer_count(7, 1) == 7 and jo.fractional_transfer_count(0, 3) == 0
+    assert jo.fractional_transfer_count(1, 9) == 1                       # progress while anything is masked
+    # without early exits it walks down exactly the fixed table, for every block length and step count
+    for Lb in range(1, 40):
+        for Tb in range(1, Lb + 1):
+            left, got = Lb, []
+            for s in range(Tb):
+                k = jo.fractional_transfer_count(left, Tb - s)
+                got.append(k)
+                left -= k
+            assert left == 0 and got == jo.transfer_counts(Lb, Tb), (Lb, Tb)
+
+
+def test_fractional_schedule_in_the_loop():
+    inf = float("inf")
+    # nothing clears the gate: same steps and same counts as the fixed table
+    fn = random_stats_fn(3)
+    a = jo.generate(None, [7, 8], 12, 8, jo.JotParams(inf, inf, 0.5, 8), M, 6, stats_fn=fn, schedule="fractional")
+    b = jo.generate(None, [7, 8], 12, 8, jo.JotParams(inf, inf, 0.5, 8), M, 6, stats_fn=fn)
+    assert a.x == b.x and [len(r.scheduled) for r in a.reports] == [2, 2, 1, 1, 2, 2, 1, 1]
+    # early exits run ahead of the pace: a hand-made model in which canvas positions 4..11 of the 12-token block
+    # 2..13 clear the threshold at the first step and also hold the highest max-probabilities.  Step 1 reveals 3
+    # (all among the 8 exits): 4 left.  The fixed table (3 per step) then reveals 3 and 1: three steps.  The
+    # fractional schedule re-divides what is still masked over the steps left: ceil(4 / 3) = 2, ceil(2 / 2) = 1,
+    # ceil(1 / 1) = 1: four steps, never more than the pace needs.
+    def stats_fn(x, A):
+        out = {}
+        for i in A:
+            sure = 4 <= i <= 11
+            out[i] = jo.RowStats(20.0 if sure else 1.0, 50 + i, 0.0, 1.0 + i * 1e-3 + (0.0 if sure else 5.0))
+        return out
+    fr = jo.generate(None, [1, 2], 12, 4, jo.JotParams(50.0, 50.0, 0.5, 8), M, None, stats_fn=stats_fn, schedule="fractional")
+    fx = jo.generate(None, [1, 2], 12, 4, jo.JotParams(50.0, 50.0, 0.5, 8), M, None, stats_fn=stats_fn)
+    assert sorted(fr.reports[0].exited) == list(range(4, 12)) and fr.reports[0].scheduled == [4, 5, 6]
+    assert [len(r.scheduled) for r in fr.reports] == [3, 2, 1, 1] and fr.steps_used == 4
+    assert [cv.count(M) for cv in fr.canvases] == [12, 4, 2, 1]
+    assert [len(r.scheduled) for r in fx.reports] == [3, 3, 1] and fx.steps_used == 3
+    # invariants under the adaptive schedule with random statistics: ends within its steps, one or more per step
+    for Lb in (None, 8):
+        tr = jo.generate(None, [5] * 6, 32, 16, jo.DREAM_DEFAULT, M, Lb, stats_fn=random_stats_fn(9), schedule="fractional")
+        assert all(t != M for t in tr.x) and tr.steps_used <= 16
+        assert all(len(r.scheduled) >= 1 for r in tr.reports)
+
+
 def test_generate_with_logits_fn_excludes_mask_token():
     V = 12
     mid = V - 1

@@ -113,6 +113,9 @@ ACCEPT_MUTATIONS = {
     "argmax ties to the highest index": ("row_stats", mut_row_stats_highest_index),
     "mask column not excluded": ("row_stats", mut_row_stats_keeps_mask_column),
     "runner-up skips exact ties": ("row_stats", mut_row_stats_distinct_runner_up),
+    "fractional schedule rounds down": ("fractional_transfer_count", lambda n, t: n // t),
+    "fractional schedule divides by one step too many": ("fractional_transfer_count", lambda n, t: -(-n // (t + 1))),
+    "fractional schedule ignores what is left": ("fractional_transfer_count", lambda n, t: 1),
     "transfer counts: remainder to the last steps": (
         "transfer_counts", lambda L, T: [L // T + (1 if s >= T - L % T else 0) for s in range(T)]),
 }
@@ -185,8 +188,10 @@ LOOP_MUTATIONS = {
     "candidates are every masked position, not the current block's": (
         "A = [i for i in range(lo, hi) if x[i] == mask_id]             # M_n",
         "A = [i for i in range(P, len(x)) if x[i] == mask_id]"),
-    "the schedule table restarts only once": ("rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[s],",
-                                              "rep = accept_freeze(x, stats, p, mask_id, lo, hi, ks[min(traj.steps_used, Tb - 1)],"),
+    "the schedule table restarts only once": ('k = ks[s] if schedule == "fixed"',
+                                              'k = ks[min(traj.steps_used, Tb - 1)] if schedule == "fixed"'),
+    "the fractional schedule counts the steps of the whole run": (
+        "fractional_transfer_count(len(A), Tb - s)", "fractional_transfer_count(len(A), steps - traj.steps_used)"),
 }
 
 
