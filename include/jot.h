@@ -58,7 +58,13 @@ int jot_last_cuda_error(void);
  * does; schedule and OR unchanged.  The compared system stages three thresholds over decoding progress
  * (7.5 / 5.0 / 2.5, Section 5.1): here the threshold is one input, which a caller stepping through
  * jot_denoise_step / jot_accept_freeze may change from step to step.  Any other gate value is refused
- * (JOT_ERR_ARG). */
+ * (JOT_ERR_ARG).
+ * schedule: how many positions the transfer schedule reveals per step inside jot_generate.  The paper leaves it
+ * to "the model's default unmasking schedule" (Section 4.2, "Interaction with transfer schedules").
+ * JOT_SCHEDULE_FIXED: block_len positions spread evenly over the block's steps, the remainder on the earliest
+ * steps.  JOT_SCHEDULE_FRACTIONAL: ceil(positions still masked in the block / steps the block has left), the
+ * adaptive rule of samplers that reveal a fraction of what remains; without early exits both give the same
+ * counts.  jot_accept_freeze takes its count as an argument and ignores the field (it must still be 0 or 1). */
 typedef struct {
     float tau_max, tau_min, gamma;
     int32_t D;
@@ -67,8 +73,10 @@ typedef struct {
     int32_t gate;            /* 0 = JOT_GATE_RATIO, 1 = JOT_GATE_MAXPROB, 2 = JOT_GATE_GLOBAL_GAP */
     float prob_threshold;    /* JOT_GATE_MAXPROB: finalise when p1 >= prob_threshold */
     float gap_threshold;     /* JOT_GATE_GLOBAL_GAP: finalise every candidate when their mean top-2 logit gap >= this */
+    int32_t schedule;        /* 0 = JOT_SCHEDULE_FIXED, 1 = JOT_SCHEDULE_FRACTIONAL (jot_generate only) */
 } jot_params;
 enum { JOT_GATE_RATIO = 0, JOT_GATE_MAXPROB = 1, JOT_GATE_GLOBAL_GAP = 2 };
+enum { JOT_SCHEDULE_FIXED = 0, JOT_SCHEDULE_FRACTIONAL = 1 };
 
 /* Geometry of the denoiser f_theta (Algorithm 1 treats it as given).  Llama-style: RMSNorm,
  * rotate-half RoPE on absolute canvas positions, grouped-query attention without any mask, SwiGLU

@@ -22,6 +22,7 @@ struct AcceptParamsDev {     // mirrors jot_params
     int32_t gate;                // 0: ratio r >= tau (Eq. 8); 1: fixed probability gate p1 >= prob_threshold;
     float prob_threshold;        // 2: global early commit, mean top-2 logit gap of the candidates >= gap_threshold
     float gap_threshold;
+    int32_t schedule;            // 0: fixed per-block table; 1: ceil(still masked / steps the block has left)
 };
 
 // Per-sequence loop state used by the generate loop (device resident).
@@ -54,6 +55,7 @@ struct AcceptArgs {
     int32_t* n_unfinished;           // device counter: += 1 per sequence that still has work (nullable)
     int lockstep;                    // generate mode under a block-wise KV cache: every sequence works on the block
                                      // [blk_lo, blk_hi) with k_transfer; the host moves all of them on together
+    int lockstep_s;                  // ... and this is the block's step index (the fractional schedule needs it)
     // generate mode, optional trace (Appendix "Confidence Dynamics"): row = the sequence's own 0-based step
     float* mean_ratio;               // [steps, B]: mean of r over the step's candidates
     int32_t* n_candidates;           // [steps, B]
@@ -153,6 +155,11 @@ accept_freeze_kernel(const AcceptArgs a, const __grid_constant__ typename Accept
         __syncthreads();
     }
     const int n_cand = n_cand_sh;
+    if (a.state && prm.schedule == 1) {
+        // adaptive schedule: the share of what is still masked that keeps the block on pace to end with its last step
+        const int steps_left = max(1, a.steps_per_block - (a.lockstep ? a.lockstep_s : st.s));
+        k = (n_cand + steps_left - 1) / steps_left;
+    }
 
     // per candidate: ratio, threshold, early-exit decision
     float r_sum = 0.f, gap_sum = 0.f;

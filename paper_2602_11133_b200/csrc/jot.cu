@@ -793,6 +793,7 @@ int launch_accept(const AcceptArgs& a, cudaStream_t st, const AcceptParamsInline
 
 bool params_ok(const jot_params* p) {
     if (!p || p->D < 1 || p->D > kMaxD) return false;
+    if (p->schedule != JOT_SCHEDULE_FIXED && p->schedule != JOT_SCHEDULE_FRACTIONAL) return false;
     if (p->gate == JOT_GATE_MAXPROB) return p->prob_threshold > 0.f && p->prob_threshold <= 1.f;
     if (p->gate == JOT_GATE_GLOBAL_GAP) return p->gap_threshold == p->gap_threshold;      // anything but NaN
     return p->gate == JOT_GATE_RATIO;
@@ -1171,7 +1172,7 @@ int jot_generate(jot_model* m, const jot_params* params, int per_seq_params, con
                 a.mask_id = m->cfg.mask_id; a.tokens = m->canvas; a.B = B; a.L = L;
                 a.top1 = m->g_top1; a.top2 = m->g_top2; a.sumexp = m->g_sumexp;
                 a.argmax = sampling ? m->g_sampled : m->g_argmax;
-                a.state = m->state; a.lockstep = 1; a.blk_lo = lo; a.blk_hi = hi;
+                a.state = m->state; a.lockstep = 1; a.lockstep_s = s; a.steps_per_block = Tb; a.blk_lo = lo; a.blk_hi = hi;
                 a.k_transfer = Lb / Tb + (s < Lb % Tb ? 1 : 0);
                 a.n_unfinished = m->ctrl + 2;
                 if (trace) {

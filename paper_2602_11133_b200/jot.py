@@ -39,17 +39,19 @@ class JotError(RuntimeError):
 
 
 GATE_RATIO, GATE_MAXPROB, GATE_GLOBAL_GAP = 0, 1, 2
+SCHEDULE_FIXED, SCHEDULE_FRACTIONAL = 0, 1
 
 
 class Params(C.Structure):
     """tau_max, tau_min, gamma, D of Algorithm 1; eps of Eq. 4."""
     _fields_ = [("tau_max", C.c_float), ("tau_min", C.c_float), ("gamma", C.c_float), ("D", C.c_int32),
                 ("eps", C.c_float), ("schedule_after_exit", C.c_int32), ("gate", C.c_int32),
-                ("prob_threshold", C.c_float), ("gap_threshold", C.c_float)]
+                ("prob_threshold", C.c_float), ("gap_threshold", C.c_float), ("schedule", C.c_int32)]
 
     def __init__(self, tau_max=90.0, tau_min=1.0, gamma=0.5, D=8, eps=1e-12, schedule_after_exit=0, gate=0,
-                 prob_threshold=0.9, gap_threshold=5.0):
-        super().__init__(tau_max, tau_min, gamma, D, eps, schedule_after_exit, gate, prob_threshold, gap_threshold)
+                 prob_threshold=0.9, gap_threshold=5.0, schedule=0):
+        super().__init__(tau_max, tau_min, gamma, D, eps, schedule_after_exit, gate, prob_threshold, gap_threshold,
+                         schedule)
 
 
 class ModelConfig(C.Structure):

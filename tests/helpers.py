@@ -103,7 +103,8 @@ def replay_trajectory(jot, model, tr: jo.Trajectory, params: jo.JotParams, mask_
         step_in_block[lo] = s + 1
         x = torch.tensor([cv], dtype=torch.int32, device="cuda")
         st = model.denoise_step(x, lo, hi, **d_bump)
-        jot.accept_freeze(jp, mask_id, x, lo, hi, ks[s], st)
+        k = ks(cv, lo, hi, s) if callable(ks) else ks[s]          # a rule (canvas, block, step in block) or a table
+        jot.accept_freeze(jp, mask_id, x, lo, hi, k, st)
         got = x.cpu()[0].tolist()
         want = tr.canvases[n + 1] if n + 1 < len(tr.canvases) else tr.x
         if got == want:
@@ -126,7 +127,7 @@ def replay_trajectory(jot, model, tr: jo.Trajectory, params: jo.JotParams, mask_
     return len(tr.canvases), excused
 
 
-def manual_generate(jot, model, prompt_row, G, T, jp, block_len, mask_id, bump=None, sampling=None):
+def manual_generate(jot, model, prompt_row, G, T, jp, block_len, mask_id, bump=None, sampling=None, fractional=False):
     """Algorithm 1 for ONE sequence driven from the host through the single-step entry points (jot_denoise_step +
     jot_accept_freeze), free-running on the GPU's own canvas.  jot_generate must give the very same tokens and
     step count: both run the same kernels on the same state, so this comparison needs no tolerance and no
@@ -151,7 +152,8 @@ def manual_generate(jot, model, prompt_row, G, T, jp, block_len, mask_id, bump=N
                 st = jot.Stats(st.top1, st.top2, st.sumexp, st.sampled)
             else:
                 st = model.denoise_step(x, lo, hi, **d_bump)
-            jot.accept_freeze(jp, mask_id, x, lo, hi, ks[s], st, n_masked)
+            k = jo.fractional_transfer_count(int((x[0, lo:hi] == mask_id).sum()), Tb - s) if fractional else ks[s]
+            jot.accept_freeze(jp, mask_id, x, lo, hi, k, st, n_masked)
             used += 1
     return x.cpu()[0].tolist(), used
 

@@ -184,6 +184,55 @@ def test_argument_validation(jot):
     model.close()
 
 
+@pytest.mark.parametrize("block_len,T", [(16, 32), (None, 16), (32, 64)])
+def test_generation_under_the_fractional_schedule(jot, block_len, T):
+    """The adaptive transfer schedule (ceil of what is still masked over the steps the block has left) inside
+    jot_generate on the tiny model with the planted bump: teacher-forced replay of the oracle's trajectory, the
+    library's loop against the host-driven loop (always), against the oracle when nothing was excused; and the
+    runs under the two schedules really differ."""
+    g = inputs.TINY
+    P, G = 32, 64
+    params = jo.LLADA_DEFAULT
+    w_cpu = inputs.model_weights(g, seed=0)
+    w_gpu = inputs.weights_to(w_cpu, "cuda")
+    prompt = inputs.prompt(0, 1, P, g.vocab, g.mask_id)
+    bump = inputs.logit_bump(9, 1, P + G, g.vocab, g.mask_id, hi=12.0)
+
+    def logits_fn(x, rows):
+        l = mo.logits(g, w_cpu, torch.tensor([x], dtype=torch.int32), rows=[(0, i) for i in rows])
+        for r, i in enumerate(rows):
+            l[r, int(bump[0][0, i])] += float(bump[1][0, i])
+        return {i: l[r].numpy() for r, i in enumerate(rows)}
+    tr = jo.generate(logits_fn, prompt[0].tolist(), G, T, params, g.mask_id, block_len, schedule="fractional")
+    tr_fixed = jo.generate(logits_fn, prompt[0].tolist(), G, T, params, g.mask_id, block_len)
+    Lb = block_len or G
+    Tb = T // (G // Lb)
+    model = jot.Model(g, w_gpu, 1, P + G)
+    rule = lambda cv, lo, hi, s: jo.fractional_transfer_count(sum(1 for i in range(lo, hi) if cv[i] == g.mask_id), Tb - s)
+    steps, excused = replay_trajectory(jot, model, tr, params, g.mask_id, rule, bump)
+    assert excused <= 2
+    jp = jot.Params(params.tau_max, params.tau_min, params.gamma, params.D, params.eps, schedule=jot.SCHEDULE_FRACTIONAL)
+    d_bump = dict(bump_id=bump[0].cuda(), bump_val=bump[1].cuda())
+    out, used, passes = model.generate(prompt.cuda(), G, T, jp, block_len, **d_bump)
+    got = out.cpu()[0].tolist()
+    assert all(t != g.mask_id for t in got) and used[0] <= T
+    from helpers import manual_generate
+    man, man_used = manual_generate(jot, model, prompt[0].tolist(), G, T, jp, block_len, g.mask_id, bump, fractional=True)
+    assert got == man and used[0] == man_used
+    if excused == 0:
+        assert used[0] == tr.steps_used and got == tr.x
+    print(f"fractional schedule, blocks of {Lb}, {Tb} steps each: {tr.steps_used} steps (fixed table: {tr_fixed.steps_used}), "
+          f"{excused} excused; oracle equality {'asserted' if excused == 0 else 'NOT asserted'}")
+    assert tr.steps_used != tr_fixed.steps_used or tr.x != tr_fixed.x or T == G      # the schedules differ once exits run ahead
+    with pytest.raises(jot.JotError):
+        model.generate(prompt.cuda(), G, T, jot.Params(schedule=7), block_len)
+    # under the block-wise KV cache (all sequences in lock-step) the same rule applies
+    model.attach_kv_cache()
+    o1 = model.generate(prompt.cuda(), G, T, jp, block_len, kv_cache=True, **d_bump)
+    assert (o1[0] != g.mask_id).all() and o1[1][0] <= T
+    model.close()
+
+
 def test_token_id_outside_the_vocabulary_is_reported_not_read(jot):
     """A token id outside [0, vocab) must come back as an argument error: the row is embedded as token 0 (no read
     leaves the embedding matrix), the status word records it, and the model works again on corrected input."""
