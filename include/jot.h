@@ -225,6 +225,26 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
                       float* d_sumexp, int32_t* d_argmax, const jot_sampling* sampling, int32_t* d_sampled,
                       void* stream);
 
+/* The same over a slice [v_lo, v_hi) of the vocabulary: top1 / argmax / top2 / sumexp of every active row taken
+ * over the token ids of the slice only (argmax is a global token id; the mask token and the bump apply when they
+ * fall inside the slice; sumexp is relative to the slice's own top1).  This is one rank's share of a
+ * vocabulary-parallel head: statistics of disjoint slices combine exactly (top1, top2, argmax) and to fp32
+ * rounding (sumexp) with jot_merge_stats, which applies to [n] arrays the associative rule the head itself uses
+ * for its vocabulary chunks: top1 = max, top2 = max of the two runner-ups and the smaller top1, sumexp rescaled
+ * to the new top1, argmax of the larger top1 (lower token id when equal).  Outputs may alias the first input.
+ * 0 <= v_lo < v_hi <= vocab; sampling is refused on a proper slice (a draw needs the whole vocabulary).  A slice
+ * that holds nothing but the excluded mask token yields top1 = -inf, sumexp = 0, argmax = INT32_MAX, the
+ * neutral element of the merge. */
+int jot_lm_head_stats_slice(jot_model* m, const void* d_hidden, const int32_t* d_tokens, int B, int L,
+                            int blk_lo, int blk_hi, int exclude_mask_token, const int32_t* d_bump_id,
+                            const float* d_bump_val, int v_lo, int v_hi, float* d_top1_logit,
+                            float* d_top2_logit, float* d_sumexp, int32_t* d_argmax,
+                            const jot_sampling* sampling, int32_t* d_sampled, void* stream);
+int jot_merge_stats(int n, const float* a_top1, const float* a_top2, const float* a_sumexp,
+                    const int32_t* a_argmax, const float* b_top1, const float* b_top2, const float* b_sumexp,
+                    const int32_t* b_argmax, float* o_top1, float* o_top2, float* o_sumexp, int32_t* o_argmax,
+                    void* stream);
+
 /* Section 4.1 Eq. 4-8 and the state update of Algorithm 1 for one step, in place on d_tokens [B, L].
  * Candidates are the positions of [blk_lo, blk_hi) that hold mask_id.  For each: confidence ratio
  * r = p1/(p2 + eps) from the statistics (Eq. 4), spatial weight over the whole canvas (Eq. 5,

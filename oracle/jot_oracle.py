@@ -101,6 +101,32 @@ def row_stats(logits: np.ndarray, mask_id: Optional[int] = None) -> RowStats:
     return RowStats(m1, i1, m2, S)
 
 
+def row_stats_slice(logits: np.ndarray, v_lo: int, v_hi: int, mask_id: Optional[int] = None) -> RowStats:
+    """row_stats over the token ids [v_lo, v_hi) only; i1 stays a global token id.  A slice with no candidate
+    (nothing but the excluded mask token) gives the neutral element (-inf, 2^31 - 1, -inf, 0)."""
+    l = np.asarray(logits, dtype=np.float64)[v_lo:v_hi].copy()
+    if mask_id is not None and v_lo <= mask_id < v_hi:
+        l[mask_id - v_lo] = -np.inf
+    if l.size == 0 or not np.isfinite(l.max()):
+        return RowStats(-math.inf, 2 ** 31 - 1, -math.inf, 0.0)
+    order = np.argsort(-l, kind="stable")
+    m1 = float(l[order[0]])
+    m2 = float(l[order[1]]) if l.size > 1 else -math.inf
+    return RowStats(m1, v_lo + int(order[0]), m2, float(np.sum(np.exp(l - m1))))
+
+
+def merge_row_stats(a: RowStats, b: RowStats) -> RowStats:
+    """Statistics of one row over two disjoint sets of token ids -> over their union (what a vocabulary-parallel
+    head does with its ranks' results).  The largest logit is the larger of the two; the runner-up is the
+    largest of the two runner-ups and the smaller of the two maxima; the sums are brought to the new maximum;
+    equal maxima resolve to the lower token id."""
+    m1 = max(a.m1, b.m1)
+    m2 = max(a.m2, b.m2, min(a.m1, b.m1))
+    S = (0.0 if a.m1 == -math.inf else a.S * math.exp(a.m1 - m1)) + (0.0 if b.m1 == -math.inf else b.S * math.exp(b.m1 - m1))
+    i1 = b.i1 if (b.m1 > a.m1 or (b.m1 == a.m1 and b.i1 < a.i1)) else a.i1
+    return RowStats(m1, i1, m2, S)
+
+
 def confidence_ratio(p1: float, p2: float, eps: float = 1e-12) -> float:
     """Eq. 4: r = p1 / (p2 + eps)."""
     return p1 / (p2 + eps)

@@ -56,6 +56,7 @@ struct GemmParams {
     const int32_t* bump_id;       // nullable, indexed by flat canvas index
     const float* bump_val;
     int mask_col;                 // column to exclude, or -1
+    int col_lo, col_hi;           // vocabulary slice [col_lo, col_hi) the statistics cover (col_hi = 0: all N columns)
     float4* partials;             // [chunks][R_pad] (m1, bitcast i1, m2, S)
     // sampling-based finalisation (inv_temperature > 0): each row also draws a token from softmax(l / T)
     float inv_temperature;
@@ -285,7 +286,9 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
             tmem_ld32(t_acc + c * 32, v);
             tmem_ld_wait();
             const int col0 = n_blk * BN + c * 32;
-            if (col0 >= p.N) break;                       // whole chunk past the vocabulary
+            const int hi_col = p.col_hi > 0 ? p.col_hi : p.N;      // the statistics cover columns [col_lo, hi_col)
+            if (col0 >= hi_col) break;                    // whole chunk past the slice
+            if (col0 + 32 <= p.col_lo) continue;          // whole chunk before it
             unsigned rel_b = (unsigned)(st.bump_col - col0);
             if (rel_b < 32u) {
 #pragma unroll
@@ -296,9 +299,9 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = (j == (int)rel_m) ? -INFINITY : v[j];
             }
-            if (col0 + 32 > p.N) {
+            if (col0 + 32 > hi_col || col0 < p.col_lo) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = (col0 + j < p.N) ? v[j] : -INFINITY;
+                for (int j = 0; j < 32; ++j) v[j] = (col0 + j < hi_col && col0 + j >= p.col_lo) ? v[j] : -INFINITY;
             }
             if (p.inv_temperature > 0.f) {
                 // Gumbel-max: argmax_v (l_v / T - ln(-ln u_v)), u_v from 23 bits of the row's counter stream
@@ -326,6 +329,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
                     st.m1 = fmaxf(st.m1, x);
                 }
             }
+            if (st.m1 == -INFINITY) continue;                // nothing but excluded columns so far: no sum yet
             // st.S = sum exp(l - st.m1): rescale what was summed against the old maximum
             const float nm = st.m1 * L2E;
             float acc_s = 0.f;
@@ -392,16 +396,21 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     const int split = (EPI == EPI_PARTIAL) ? p.split_k : 1;
     int total_tiles = num_m * num_n * split;
     int chunk = 0;
+    // EPI_STATS: only the tiles that touch the vocabulary slice are visited
+    const int stats_hi = (EPI == EPI_STATS && p.col_hi > 0) ? p.col_hi : p.N;
+    const int tile_lo = (EPI == EPI_STATS) ? p.col_lo / BN : 0;
+    const int num_nt = (EPI == EPI_STATS) ? (stats_hi + BN - 1) / BN - tile_lo : num_n;
     if (EPI == EPI_STATS) {
         int R = *p.d_R, n_rb, n_ch;
-        stats_partition(R, gridDim.x, num_n, &n_rb, &n_ch);
+        stats_partition(R, gridDim.x, num_nt, &n_rb, &n_ch);
         chunk = n_rb > 0 ? blockIdx.x / n_rb : 0;
         if (n_rb == 0 || chunk >= n_ch) {
             n_count = 0;
         } else {
             m_blk0 = blockIdx.x % n_rb;
-            n_first = (int)((long long)chunk * num_n / n_ch);
-            n_count = (int)((long long)(chunk + 1) * num_n / n_ch) - n_first;
+            n_first = (int)((long long)chunk * num_nt / n_ch);
+            n_count = (int)((long long)(chunk + 1) * num_nt / n_ch) - n_first;
+            n_first += tile_lo;
         }
         total_tiles = n_count;
     }

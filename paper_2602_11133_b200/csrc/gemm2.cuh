@@ -85,15 +85,19 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
     int m_blk0 = 0, n_first = 0, chunk = 0;
     bool stats_row_block_valid = false;
     if (EPI == EPI_STATS) {
+        // only the tiles that touch the vocabulary slice [col_lo, col_hi) are visited
+        const int stats_hi = p.col_hi > 0 ? p.col_hi : p.N;
+        const int tile_lo = p.col_lo / BN, num_nt = (stats_hi + BN - 1) / BN - tile_lo;
         int n_rb, n_pr, n_ch;
-        stats_partition_pair(*p.d_R, n_clusters, num_n, &n_rb, &n_pr, &n_ch);
+        stats_partition_pair(*p.d_R, n_clusters, num_nt, &n_rb, &n_pr, &n_ch);
         chunk = n_pr > 0 ? cluster_id / n_pr : 0;
         total_tiles = 0;
         if (n_pr > 0 && chunk < n_ch) {
             m_blk0 = 2 * (cluster_id % n_pr) + rank;
             stats_row_block_valid = m_blk0 < n_rb;
-            n_first = (int)((long long)chunk * num_n / n_ch);
-            total_tiles = (int)((long long)(chunk + 1) * num_n / n_ch) - n_first;
+            n_first = (int)((long long)chunk * num_nt / n_ch);
+            total_tiles = (int)((long long)(chunk + 1) * num_nt / n_ch) - n_first;
+            n_first += tile_lo;
         }
     }
     auto tile_at = [&](int it, int& m_blk, int& n_blk) -> bool {

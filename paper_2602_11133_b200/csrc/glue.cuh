@@ -322,6 +322,25 @@ __global__ void __launch_bounds__(128) merge_stats_kernel(const float4* __restri
     }
 }
 
+// Statistics of the same rows over two disjoint parts of the vocabulary -> statistics over their union, element by
+// element over [n] arrays (the rule merge_stats_kernel applies to the chunks of one launch): what a rank does with
+// the tuples its peers computed on their vocabulary slices.  out may alias a.
+__global__ void merge_stat_arrays_kernel(int n, const float* __restrict__ a1, const float* __restrict__ a2,
+                                         const float* __restrict__ aS, const int32_t* __restrict__ ai,
+                                         const float* __restrict__ b1, const float* __restrict__ b2,
+                                         const float* __restrict__ bS, const int32_t* __restrict__ bi, float* o1,
+                                         float* o2, float* oS, int32_t* oi) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const StatTuple t = merge_tuples(StatTuple{a1[i], a2[i], aS[i], ai[i]}, StatTuple{b1[i], b2[i], bS[i], bi[i]});
+    o1[i] = t.m1;
+    o2[i] = t.m2;
+    oS[i] = t.S;
+    oi[i] = t.i1;
+}
+
 // Sequences that still have work, in ascending order: seq_map[slot] = b, the remaining slots -1,
 // *n_active = count.  One warp.
 __global__ void build_seq_map_kernel(const SeqState* __restrict__ state, int B, int n_blocks,

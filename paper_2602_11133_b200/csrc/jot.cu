@@ -676,7 +676,7 @@ struct HeadSampling {
 
 int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, const float* bump_val, float* top1,
                       float* top2, float* sumexp, int32_t* argmax, int M, cudaStream_t st,
-                      const HeadSampling* hs = nullptr) {
+                      const HeadSampling* hs = nullptr, int v_lo = 0, int v_hi = 0) {
     const jot_model_config& c = m->cfg;
     if (M <= 0) return JOT_OK;                       // an empty block range has no active rows
     if (M > jot_max_active_rows(m->di->sms)) return JOT_ERR_SHAPE;   // every row block needs a CTA (pair) of its own
@@ -685,6 +685,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
     p.d_R = m->ctrl + 1; p.rows = m->rows_out; p.bump_id = bump_id; p.bump_val = bump_val;
     p.mask_col = exclude_mask ? c.mask_id : -1;
     p.partials = m->partials; p.R_pad = m->R_cap;
+    p.col_lo = v_lo; p.col_hi = v_hi;                 // (0, 0): the whole vocabulary
     const bool sampling = hs && hs->temperature > 0.f;
     if (sampling) {
         p.inv_temperature = 1.f / hs->temperature; p.sample_seed = hs->seed; p.d_seq_steps = hs->d_seq_steps;
@@ -707,7 +708,7 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
             JOT_TRY((launch_pair_t<EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
         }
     }
-    const int n_vt = (c.vocab + bn - 1) / bn;
+    const int n_vt = ((v_hi > 0 ? v_hi : c.vocab) + bn - 1) / bn - v_lo / bn;     // tiles that touch the slice
     ProfScope ps(m, JOT_PROF_MERGE, st);
     launch_k(merge_stats_kernel, dim3((M + 3) / 4), dim3(128), 0, st, m->partials, m->R_cap, grid, n_vt, mode == 2 ? 1 : 0,
              m->rows_out, m->ctrl + 1, top1, top2, sumexp, argmax, sampling ? m->partials2 : nullptr,
@@ -963,8 +964,31 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
                       int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val, float* d_top1,
                       float* d_top2, float* d_sumexp, int32_t* d_argmax, const jot_sampling* sampling,
                       int32_t* d_sampled, void* stream) {
+    return jot_lm_head_stats_slice(m, d_hidden, d_tokens, B, L, blk_lo, blk_hi, exclude_mask_token, d_bump_id, d_bump_val,
+                                   0, m ? m->cfg.vocab : 0, d_top1, d_top2, d_sumexp, d_argmax, sampling, d_sampled, stream);
+}
+
+int jot_merge_stats(int n, const float* a_top1, const float* a_top2, const float* a_sumexp, const int32_t* a_argmax,
+                    const float* b_top1, const float* b_top2, const float* b_sumexp, const int32_t* b_argmax,
+                    float* o_top1, float* o_top2, float* o_sumexp, int32_t* o_argmax, void* stream) {
+    if (n < 0 || !a_top1 || !a_top2 || !a_sumexp || !a_argmax || !b_top1 || !b_top2 || !b_sumexp || !b_argmax || !o_top1 ||
+        !o_top2 || !o_sumexp || !o_argmax)
+        return JOT_ERR_ARG;
+    if (n == 0) return JOT_OK;
+    launch_k(merge_stat_arrays_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, (cudaStream_t)stream, n, a_top1, a_top2,
+             a_sumexp, a_argmax, b_top1, b_top2, b_sumexp, b_argmax, o_top1, o_top2, o_sumexp, o_argmax);
+    return launch_check();
+}
+
+int jot_lm_head_stats_slice(jot_model* m, const void* d_hidden, const int32_t* d_tokens, int B, int L, int blk_lo,
+                            int blk_hi, int exclude_mask_token, const int32_t* d_bump_id, const float* d_bump_val,
+                            int v_lo, int v_hi, float* d_top1, float* d_top2, float* d_sumexp, int32_t* d_argmax,
+                            const jot_sampling* sampling, int32_t* d_sampled, void* stream) {
     JOT_TRY(check_step_args(m, d_tokens, B, L, blk_lo, blk_hi, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax));
     if (!d_hidden) return JOT_ERR_ARG;
+    if (v_lo < 0 || v_hi > m->cfg.vocab || v_lo >= v_hi) return JOT_ERR_ARG;
+    const bool whole = v_lo == 0 && v_hi == m->cfg.vocab;
+    if (!whole && sampling && sampling->temperature > 0.f) return JOT_ERR_ARG;   // a draw needs the whole vocabulary
     HeadSampling hs;
     JOT_TRY(head_sampling_from(sampling, d_sampled, &hs));
     cudaStream_t st = (cudaStream_t)stream;
@@ -979,7 +1003,7 @@ int jot_lm_head_stats(jot_model* m, const void* d_hidden, const int32_t* d_token
         JOT_TRY(launch_check());
     }
     JOT_TRY(lm_head_from_hsel(m, exclude_mask_token, d_bump_id, d_bump_val, d_top1, d_top2, d_sumexp, d_argmax,
-                              B * (blk_hi - blk_lo), st, &hs));
+                              B * (blk_hi - blk_lo), st, &hs, whole ? 0 : v_lo, whole ? 0 : v_hi));
     return m->sync_steps ? read_status(m, st) : JOT_OK;
 }
 

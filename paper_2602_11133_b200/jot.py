@@ -22,6 +22,7 @@ EXPORTS = [
     "jot_launch_count", "jot_profile", "jot_profile_read", "jot_gemm_bf16_noalloc",
     "jot_selftest_wait_expiry", "jot_kv_cache_bytes", "jot_attach_kv_cache", "jot_denoise_step_cached",
     "jot_max_active_rows", "jot_lm_head_partition", "jot_set_sync", "jot_read_status",
+    "jot_lm_head_stats_slice", "jot_merge_stats",
 ]
 
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -114,6 +115,10 @@ def _lib():
                      C.c_void_p, C.c_void_p, C.POINTER(Sampling), C.c_void_p, C.c_void_p]
         lib.jot_denoise_step.argtypes = [C.c_void_p, C.c_void_p] + step_args
         lib.jot_lm_head_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + step_args
+        lib.jot_lm_head_stats_slice.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                C.c_void_p, C.POINTER(Sampling), C.c_void_p, C.c_void_p]
+        lib.jot_merge_stats.argtypes = [C.c_int] + [C.c_void_p] * 13
         lib.jot_kv_cache_bytes.restype = C.c_size_t
         lib.jot_kv_cache_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int, C.c_int]
         lib.jot_attach_kv_cache.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
@@ -324,6 +329,24 @@ class Model:
                "jot_lm_head_stats")
         return out
 
+    def lm_head_stats_slice(self, hidden: torch.Tensor, tokens: torch.Tensor, blk_lo: int, blk_hi: int, v_lo: int,
+                            v_hi: int, out: Optional[Stats] = None, exclude_mask_token: bool = True,
+                            bump_id: Optional[torch.Tensor] = None, bump_val: Optional[torch.Tensor] = None) -> Stats:
+        """Statistics of the active rows over the vocabulary slice [v_lo, v_hi) only (one rank's share of a
+        vocabulary-parallel head)."""
+        B, L = tokens.shape
+        if hidden.shape != (B * L, self.cfg.d_model):
+            raise ValueError("hidden must be [B*L, d_model]")
+        out = out or Stats.empty(B, L, tokens.device)
+        _check(_lib().jot_lm_head_stats_slice(self.handle, _ptr(hidden, torch.bfloat16, "hidden"),
+                                              _ptr(tokens, torch.int32, "tokens"), B, L, blk_lo, blk_hi,
+                                              int(exclude_mask_token), _ptr(bump_id, torch.int32, "bump_id"),
+                                              _ptr(bump_val, torch.float32, "bump_val"), v_lo, v_hi, out.top1.data_ptr(),
+                                              out.top2.data_ptr(), out.sumexp.data_ptr(), out.argmax.data_ptr(), None,
+                                              None, _stream()),
+               "jot_lm_head_stats_slice")
+        return out
+
     # ---- Algorithm 1 ----------------------------------------------------------------------------
     def generate(self, prompt: torch.Tensor, gen_len: int, steps: int, params, block_len: Optional[int] = None,
                  exclude_mask_token: bool = True, bump_id: Optional[torch.Tensor] = None,
@@ -382,6 +405,19 @@ def accept_freeze(params, mask_id: int, tokens: torch.Tensor, blk_lo: int, blk_h
                                     _ptr(exit_reason, torch.uint8, "exit_reason"),
                                     _ptr(exit_step, torch.int16, "exit_step"), step_index, _stream()),
            "jot_accept_freeze")
+
+
+def merge_stats(a: Stats, b: Stats, out: Optional[Stats] = None) -> Stats:
+    """Statistics of the same positions over two disjoint vocabulary slices -> over their union (device kernel)."""
+    out = out or Stats(torch.empty_like(a.top1), torch.empty_like(a.top2), torch.empty_like(a.sumexp),
+                       torch.empty_like(a.argmax))
+    n = a.top1.numel()
+    args = []
+    for s in (a, b, out):
+        args += [_ptr(s.top1, torch.float32, "top1"), _ptr(s.top2, torch.float32, "top2"),
+                 _ptr(s.sumexp, torch.float32, "sumexp"), _ptr(s.argmax, torch.int32, "argmax")]
+    _check(_lib().jot_merge_stats(n, *args, _stream()), "jot_merge_stats")
+    return out
 
 
 def gemm_bf16(a: torch.Tensor, w: torch.Tensor, residual: Optional[torch.Tensor] = None,

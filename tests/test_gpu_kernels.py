@@ -313,6 +313,73 @@ def test_lm_head_mask_token_and_ties(jot):
     model.close()
 
 
+# ---------------------------------------------------------------- vocabulary slices (one rank's share of the head)
+@pytest.mark.parametrize("B,P,G,d,V,cuts", [
+    (1, 32, 64, 256, 4096, (2048,)),                    # two equal slices, narrow-tile schedule
+    (2, 40, 200, 512, 5000, (1280, 2560, 3840)),        # four slices, ragged vocabulary tail, two row blocks
+    (8, 128, 256, 1024, 12800, (6400,)),                # CTA-pair schedule
+    (2, 16, 100, 256, 4096, (1000, 3001)),              # cuts that are not tile multiples
+])
+def test_vocabulary_slices_merge_to_the_full_head(jot, B, P, G, d, V, cuts):
+    """The head over disjoint vocabulary slices, merged on the device by the head's own rule, equals the head over
+    the whole vocabulary: top-1, runner-up and argmax exactly, the sum to fp32 rounding; each slice equals the
+    oracle's statistics of that slice."""
+    from paper_2602_11133_b200 import vocab_parallel as vp
+    mask_id = V - 7
+    case = inputs.lm_head_case(6, B, P, G, d, V, mask_id, device="cuda")
+    model = lm_head_model(jot, d, V, mask_id, case.w, B, P + G)
+    L = P + G
+    kw = dict(bump_id=case.bump_id, bump_val=case.bump_val)
+    full = model.lm_head_stats(case.hidden, case.tokens, P, L, **kw)
+    bounds = [0] + list(cuts) + [V]
+    parts = [model.lm_head_stats_slice(case.hidden, case.tokens, P, L, a, b, **kw) for a, b in zip(bounds, bounds[1:])]
+    acc = parts[0]
+    for nxt in parts[1:]:
+        acc = jot.merge_stats(acc, nxt)
+    tok = case.tokens.cpu()
+    active = (tok == mask_id)
+    active[:, :P] = False
+    assert int(active.sum()) > 0
+    a = active.cuda()
+    assert torch.equal(acc.top1[a], full.top1[a]) and torch.equal(acc.top2[a], full.top2[a])
+    assert torch.equal(acc.argmax[a], full.argmax[a])
+    assert torch.allclose(acc.sumexp[a], full.sumexp[a], rtol=3e-5, atol=0)      # fp32 sums of approximate exponentials in another order
+    # the packed 16-byte tuples survive the round trip of the exchange format
+    t = vp.unpack_tuples(vp.pack_tuples(acc.top1, acc.top2, acc.sumexp, acc.argmax))
+    assert torch.equal(t[0], acc.top1) and torch.equal(t[3], acc.argmax)
+    # a few rows of every slice against the oracle's slice statistics
+    rows = [(b, i) for b in range(B) for i in range(P, L) if bool(active[b, i])][:: max(1, int(active.sum()) // 6)][:6]
+    flat = torch.tensor([b * L + i for b, i in rows])
+    logits = mo.lm_head_logits(case.hidden.cpu()[flat], case.w.cpu(), case.bump_id.cpu().view(-1)[flat],
+                               case.bump_val.cpu().view(-1)[flat])
+    for (lo, hi), st in zip(zip(bounds, bounds[1:]), parts):
+        want = [jo.row_stats_slice(logits[r].numpy(), lo, hi, mask_id) for r in range(len(rows))]
+        pick = lambda t: t.cpu().view(-1)[flat].numpy()
+        compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), want, rel=1e-3)
+    with pytest.raises(jot.JotError):
+        model.lm_head_stats_slice(case.hidden, case.tokens, P, L, 10, 10, **kw)
+    with pytest.raises(jot.JotError):
+        model.lm_head_stats_slice(case.hidden, case.tokens, P, L, 0, V + 1, **kw)
+    model.close()
+
+
+def test_vocabulary_slice_with_nothing_but_the_mask_token(jot):
+    d, V, mask_id, B, L = 64, 512, 100, 1, 128
+    w = (torch.randn(V, d) * 0.1).bfloat16()
+    hidden = torch.randn(B * L, d).bfloat16()
+    tokens = torch.full((B, L), mask_id, dtype=torch.int32)
+    model = lm_head_model(jot, d, V, mask_id, w.cuda(), B, L)
+    e = model.lm_head_stats_slice(hidden.cuda(), tokens.cuda(), 0, L, 100, 101)
+    assert (e.top1 == -float("inf")).all() and (e.sumexp == 0).all() and (e.argmax == 2 ** 31 - 1).all()
+    rest_a = model.lm_head_stats_slice(hidden.cuda(), tokens.cuda(), 0, L, 0, 100)
+    rest_b = model.lm_head_stats_slice(hidden.cuda(), tokens.cuda(), 0, L, 101, V)
+    full = model.lm_head_stats(hidden.cuda(), tokens.cuda(), 0, L)
+    acc = jot.merge_stats(jot.merge_stats(rest_a, e), rest_b)
+    assert torch.equal(acc.top1, full.top1) and torch.equal(acc.argmax, full.argmax) and torch.equal(acc.top2, full.top2)
+    assert torch.allclose(acc.sumexp, full.sumexp, rtol=3e-5)
+    model.close()
+
+
 # ---------------------------------------------------------------- sampling-based finalisation (Section 4.1)
 @pytest.mark.parametrize("B,P,G,d,V,T", [
     (1, 32, 64, 256, 4096, 1.0),          # one narrow-tile chunk schedule

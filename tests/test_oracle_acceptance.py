@@ -117,6 +117,35 @@ def test_row_stats_brute_force_tiny_vocab():
             assert jo.confidence_ratio(st.p1, st.p2) < 1.0
 
 
+def test_slice_statistics_merge_to_the_whole_row():
+    # brute force on tiny vocabularies with ties and an excluded column: any cut into 1..4 slices, merged in any
+    # order and association, gives the single-pass statistics (top-1, runner-up and argmax exactly, the sum to
+    # rounding)
+    rng = random.Random(7)
+    for trial in range(300):
+        V = rng.randrange(2, 14)
+        l = np.array([rng.choice([-1.0, 0.0, 0.5, 2.0, 2.0, 3.25]) for _ in range(V)])
+        mask = rng.choice([None, rng.randrange(V)])
+        if mask is not None and V == 2:
+            continue
+        want = jo.row_stats(l, mask)
+        cuts = sorted(rng.sample(range(1, V), min(rng.randrange(0, 4), V - 1)))
+        parts = [jo.row_stats_slice(l, a, b, mask) for a, b in zip([0] + cuts, cuts + [V])]
+        rng.shuffle(parts)
+        while len(parts) > 1:                                    # random association
+            k = rng.randrange(len(parts) - 1)
+            parts[k:k + 2] = [jo.merge_row_stats(parts[k], parts[k + 1])]
+        got = parts[0]
+        assert (got.m1, got.i1, got.m2) == (want.m1, want.i1, want.m2), (l, mask, cuts)
+        assert got.S == pytest.approx(want.S, rel=1e-12)
+    # the neutral element: a slice that holds only the excluded token changes nothing
+    e = jo.row_stats_slice(np.array([1.0, 5.0, 2.0]), 1, 2, mask_id=1)
+    a = jo.row_stats_slice(np.array([1.0, 5.0, 2.0]), 0, 1)
+    assert e.m1 == -math.inf and e.S == 0.0
+    m = jo.merge_row_stats(a, e)
+    assert (m.m1, m.i1, m.m2, m.S) == (a.m1, a.i1, a.m2, a.S) and jo.merge_row_stats(e, a).i1 == a.i1
+
+
 def test_ratio_temperature_invariance_of_the_definition():
     # r uses un-tempered logits, so it is exp(gap) whatever else is in the row
     l = np.array([0.3, 5.0, 1.0, -2.0])

@@ -113,6 +113,19 @@ ACCEPT_MUTATIONS = {
     "argmax ties to the highest index": ("row_stats", mut_row_stats_highest_index),
     "mask column not excluded": ("row_stats", mut_row_stats_keeps_mask_column),
     "runner-up skips exact ties": ("row_stats", mut_row_stats_distinct_runner_up),
+    "merge: runner-up forgets the smaller maximum": (
+        "merge_row_stats", lambda a, b: jo.RowStats(max(a.m1, b.m1), b.i1 if (b.m1 > a.m1 or (b.m1 == a.m1 and b.i1 < a.i1)) else a.i1,
+                                                    max(a.m2, b.m2),
+                                                    (0.0 if a.m1 == -math.inf else a.S * math.exp(a.m1 - max(a.m1, b.m1))) +
+                                                    (0.0 if b.m1 == -math.inf else b.S * math.exp(b.m1 - max(a.m1, b.m1))))),
+    "merge: sums added without rescaling": (
+        "merge_row_stats", lambda a, b: jo.RowStats(max(a.m1, b.m1), b.i1 if (b.m1 > a.m1 or (b.m1 == a.m1 and b.i1 < a.i1)) else a.i1,
+                                                    max(a.m2, b.m2, min(a.m1, b.m1)), a.S + b.S)),
+    "merge: equal maxima resolve to the later slice": (
+        "merge_row_stats", lambda a, b: jo.RowStats(max(a.m1, b.m1), b.i1 if b.m1 >= a.m1 else a.i1,
+                                                    max(a.m2, b.m2, min(a.m1, b.m1)),
+                                                    (0.0 if a.m1 == -math.inf else a.S * math.exp(a.m1 - max(a.m1, b.m1))) +
+                                                    (0.0 if b.m1 == -math.inf else b.S * math.exp(b.m1 - max(a.m1, b.m1))))),
     "fractional schedule rounds down": ("fractional_transfer_count", lambda n, t: n // t),
     "fractional schedule divides by one step too many": ("fractional_transfer_count", lambda n, t: -(-n // (t + 1))),
     "fractional schedule ignores what is left": ("fractional_transfer_count", lambda n, t: 1),
