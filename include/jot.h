@@ -56,7 +56,7 @@ int jot_last_cuda_error(void);
  * the mean over the sequence's candidates (masked positions of the current block) of the top-2 logit gap
  * top1 - top2 is compared with gap_threshold (inclusive, in fp32) and either every candidate exits or none
  * does; schedule and OR unchanged.  The compared system stages three thresholds over decoding progress
- * (7.5 / 5.0 / 2.5, Section 5.1): here the threshold is one input, which a caller stepping through
+ * (7.5 / 5.0 / 2.5, Section 6.1 "Experimental Setup"): here the threshold is one input, which a caller stepping through
  * jot_denoise_step / jot_accept_freeze may change from step to step.  Any other gate value is refused
  * (JOT_ERR_ARG).
  * schedule: how many positions the transfer schedule reveals per step inside jot_generate.  The paper leaves it
@@ -268,7 +268,7 @@ int jot_accept_freeze(const jot_params* params, int per_seq_params, int32_t mask
  * contain mask_id; ids must lie in [0, vocab), else JOT_ERR_ARG).  Each sequence keeps its own block pointer and step counter and idles once
  * finished; the loop ends when no sequence has a masked position left, or after `steps` iterations.
  * Outputs: d_out_tokens [B, P + gen_len] (device); h_steps_used [B] (host) = denoising steps each
- * sequence actually ran (step speed-up = steps / steps_used, Section 5.1); optional
+ * sequence actually ran (step speed-up = steps / steps_used, Section 6.1 "Experimental Setup"); optional
  * h_forward_passes (host, one int) = batched forward passes executed.
  * d_bump_id / d_bump_val: as in jot_denoise_step, indexed [B, P + gen_len], fixed across steps.
  * trace (nullable, any member nullable): what the paper's analysis plots are made of.  Device arrays,

@@ -52,7 +52,7 @@ class JotParams:
     global early-commit rule the paper contrasts it with (Section 2: "once the top-2 confidence gap exceeds a
     threshold, all remaining masked positions are finalized simultaneously"): the mean over the candidates of
     the top-2 logit gap m1 - m2 is tested against gap_threshold and either every candidate exits or none does.
-    The compared system stages three thresholds over decoding progress (7.5 / 5.0 / 2.5, Section 5.1); here
+    The compared system stages three thresholds over decoding progress (7.5 / 5.0 / 2.5, Section 6.1 "Experimental Setup"); here
     the threshold is one input that a caller may change from step to step."""
     tau_max: float = 90.0
     tau_min: float = 1.0

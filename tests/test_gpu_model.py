@@ -56,6 +56,13 @@ def test_denoise_step_matches_oracle(jot, name, B, P, G, p_mask):
     print(f"{name}: {n} rows, {near} with top-2 gap < {GAP_TOL}, max |top1 err| "
           f"{max(abs(a - s.m1) for a, s in zip(pick(st.top1), want)):.2e}")
     assert near <= max(2, n // 20)
+    # the same against the oracle without any bf16 rounding of activations: the plain float64 network
+    plain = oracle_stats_for_rows(mo.logits(g, w_cpu, tokens, rows=rows, round_activations=False), g.mask_id)
+    n2, near2 = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), plain, rel=REL_TOL,
+                              gap_from_tolerance=True)
+    err = max(abs(a - s.m1) / max(abs(s.m1), 1.0) for a, s in zip(pick(st.top1), plain))
+    print(f"{name}: against the unrounded float64 oracle: max relative top-1 logit error {err:.2e} (tolerance {REL_TOL:g}), "
+          f"{near2} of {n2} rows inside the argmax margin")
     model.close()
 
 

@@ -60,7 +60,7 @@ def test_window_radius_and_edges():
 
 
 def test_no_spatial_special_case():
-    # tau_max == tau_min: the threshold is the same everywhere (threshold-only ablation, Section 5.2)
+    # tau_max == tau_min: the threshold is the same everywhere (Section 6.3 "Threshold Ablation")
     p = jo.JotParams(90.0, 90.0, 0.5, 8)
     x = canvas("rrrrmmmmmmmmrmmmrr")
     assert {jo.position_threshold(x, i, M, p) for i in range(len(x)) if x[i] == M} == {90.0}
@@ -301,7 +301,7 @@ def test_generate_threshold_zero_finishes_one_step_per_block():
     assert tr.steps_used == 1
     tr = jo.generate(None, prompt, 32, 32, jo.JotParams(0.0, 0.0, 0.5, 8), M, 8, stats_fn=random_stats_fn(2))
     assert tr.steps_used == 4
-    # step-speedup = configured / actual steps (Section 5.1)
+    # step-speedup = configured / actual steps (Section 6.1 "Experimental Setup")
     assert 32 / tr.steps_used == 8.0
 
 
@@ -406,7 +406,7 @@ def test_generate_with_logits_fn_excludes_mask_token():
 
 
 def test_reversal_budget_number():
-    # Section 5 (theory): 2 * 256 / (1 + 90) is "about 5.6"
+    # Section 5 "Why Early Exit Preserves Quality": 2 * 256 / (1 + 90) is "about 5.6"
     assert 2 * 256 / 91 == pytest.approx(5.6, abs=0.05)
 
 
