@@ -16,6 +16,12 @@ path keeps in bf16 are rounded to bf16 here at the same named points, and nowher
   output; each residual sum (projection + residual, rounded once); silu(gate)*up (from unrounded
   gate and up); logits are float64 and never rounded.
 `round_activations=False` drops every one of those roundings (pure float64 reference).
+The attention probabilities are rounded relative to the exact row maximum, which is the plain definition
+of a numerically safe softmax.  A device path that keeps an online reference maximum (one pass over the keys,
+the reference possibly lagging the true maximum by a bounded factor) rounds exp(s - reference) instead: bf16
+rounding is relative, so each probability then differs from the one here by at most one bf16 ulp (2^-8
+relative) and the normalised output by far less than the stated logit tolerance; the oracle keeps the
+definition and does not imitate any blocking of the keys.
 
 Pinned by tests against closed forms (RoPE rotation, attention row sums, permutation behaviour) and
 against an independent restatement built from torch.nn.functional routines; the float64/bf16
