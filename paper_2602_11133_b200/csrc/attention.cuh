@@ -1,19 +1,22 @@
 // Bidirectional (unmasked) grouped-query softmax attention on tcgen05 / tensor memory, fed by TMA.
 //
 // Persistent CTAs walk over work items (query block of 128 rows, query head, sequence), ordered so that the
-// CTAs running side by side share K and V of one KV head in L2.  For one item the keys are visited in blocks
-// of 128, twice:
-//   pass 1   S = Q K^T per key block -> exact row maximum m
-//   pass 2   S again; P = bf16(exp((S - m) / sqrt(hd))) written to shared memory as the A operand of
-//            O += P V ; row sum l accumulated in fp32 from the unrounded exponentials
-// and finally O / l is written as bf16.  Knowing m before any P is formed means the accumulator in tensor
-// memory is never rescaled and P is rounded against the true maximum.
+// CTAs running side by side share K and V of one KV head in L2.  For one item the keys are visited ONCE, in
+// blocks of 128:
+//   S = Q K^T for the block (tensor memory, double buffered: S(j+1) is computed while block j is in softmax)
+//   P = bf16(exp((S - m_ref) / sqrt(hd))) written to shared memory as the A operand of  O += P V
+// Two threads share a query row, each owning 64 of the block's 128 key columns, and each keeps ITS OWN running
+// reference maximum m_ref, row sum and output accumulator (O_left and O_right in tensor memory, fed by the two
+// 64-key halves of P V): no exchange between the two threads per block, only once per item, when the halves
+// are combined as (O_l 2^(m_l - m) + O_r 2^(m_r - m)) / (l_l 2^(m_l - m) + l_r 2^(m_r - m)).
+// The reference maximum is lazy: it is raised only when a block's maximum exceeds it by more than 2^8
+// (probabilities up to 256 are exact enough in bf16 and fp32); the owner thread then rescales its row of its
+// accumulator in tensor memory (tcgen05.ld / st, between the P V of the previous block and that of this one) and
+// its running sum.  With well-behaved scores that happens in the first block only, where there is nothing to rescale.
 //
-//   warp 0 (one lane)  TMA producer: Q per item, K blocks (both passes), V^T blocks (pass 2)
-//   warp 1 (one lane)  MMA issuer; S double buffered in tensor memory (S(g+1) overlaps softmax(g)), O double
-//                      buffered across items (the output of item i drains while item i+1 accumulates)
-//   warps 2..9         softmax: two threads per query row (TMEM lane), each owning 64 of the 128 key columns
-//                      of a block and half of the output columns; row max and row sum meet in shared memory
+//   warp 0 (one lane)  TMA producer: Q per item, then K and V^T block by block
+//   warp 1 (one lane)  MMA issuer
+//   warps 2..9         softmax: thread (r, hf) owns query row r (TMEM lane) and key columns [64 hf, 64 hf + 64)
 //
 // Layouts: qkv [B*L, (nq + 2 nkv) * hd] after RoPE (3-D tensor map (col, position, sequence) so that a
 // block never reads across a sequence boundary: out-of-range positions read as zero); V transposed
@@ -47,6 +50,16 @@ struct AttnSmem {
     static constexpr int DYN_BYTES = Q_BYTES + 2 * K_BYTES + 2 * V_BYTES + P_BYTES + 1024;
 };
 
+#ifdef JOT_ATTN_TRACE
+// Cycles one softmax thread of every CTA spent in each phase of the key loop; only in instrumented builds.
+__device__ long long g_attn_trace[256 * 8];
+#define ATTN_T(var) const long long var = clock64()
+#define ATTN_ACC(slot, a, b) do { if (threadIdx.x == 64) g_attn_trace[(blockIdx.x & 255) * 8 + (slot)] += (b) - (a); } while (0)
+#else
+#define ATTN_T(var) do { } while (0)
+#define ATTN_ACC(slot, a, b) do { } while (0)
+#endif
+
 template <int HD>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, const __grid_constant__ CUtensorMap tmVt) {
@@ -55,7 +68,8 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t IDESC_S = umma_idesc_bf16(128, 128);
     constexpr uint32_t IDESC_O = umma_idesc_bf16(128, HD);
-    constexpr uint32_t O_COL = 256;            // S buffers at columns 0 and 128, O buffers at 256 and 384
+    constexpr uint32_t O_COL = 256;            // S buffers at columns 0 and 128, O_left at 256, O_right at 384
+    constexpr float kRaise = 8.f;              // the reference maximum follows a block maximum more than 2^8 above it
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -64,7 +78,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
     uint8_t* sV = sK + 2 * SM::K_BYTES;      // 2 stages
     uint8_t* sP = sV + 2 * SM::V_BYTES;
     __shared__ uint64_t q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full,
-        p_empty, o_full[2], o_empty[2], xmax_bar, xsum_bar;
+        p_empty, o_full, o_empty, x_bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ float x_max[2][128], x_sum[2][128];
@@ -86,13 +100,12 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
             mbar_init(&v_empty[i], 1);
             mbar_init(&s_full[i], 1);
             mbar_init(&s_empty[i], 8);
-            mbar_init(&o_full[i], 1);
-            mbar_init(&o_empty[i], 8);
         }
-        mbar_init(&p_full, kAttnSoftmaxThreads);
+        mbar_init(&p_full, kAttnSoftmaxThreads / 32);      // one arrival per softmax warp
         mbar_init(&p_empty, 1);
-        mbar_init(&xmax_bar, kAttnSoftmaxThreads);
-        mbar_init(&xsum_bar, kAttnSoftmaxThreads);
+        mbar_init(&o_full, 1);
+        mbar_init(&o_empty, 8);
+        mbar_init(&x_bar, kAttnSoftmaxThreads / 32);
         fence_barrier_init();
         fence_proxy_async_smem();
         tma_prefetch_desc(&tmQKV);
@@ -120,7 +133,7 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
 
     if (warp == 0) {
         if (lane == 0) {
-            uint32_t gk = 0, gv = 0;     // running counts of K loads (= S products) and V loads (= P.V products)
+            uint32_t g = 0;              // running count of key blocks (K and V loads, S and P.V products)
             int it = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
@@ -133,76 +146,70 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
                     tma_load_3d(sQ + kb * 16384, &tmQKV, &q_full, q_col + kb * 64, p.q_lo + q_blk * 128, b);
-                for (int g = 0; g < 2 * nkb; ++g, ++gk) {
-                    const int j = g % nkb, st = gk & 1;
-                    if (!mbar_wait(&k_empty[st], ((gk >> 1) & 1) ^ 1, abortp)) { ok = false; break; }
+                for (int j = 0; j < nkb; ++j, ++g) {
+                    const int st = g & 1;
+                    if (!mbar_wait(&k_empty[st], ((g >> 1) & 1) ^ 1, abortp)) { ok = false; break; }
                     mbar_arrive_expect_tx(&k_full[st], SM::K_BYTES);
 #pragma unroll
                     for (int kb = 0; kb < KB; ++kb)
                         tma_load_3d(sK + st * SM::K_BYTES + kb * 16384, &tmQKV, &k_full[st], k_col + kb * 64, j * 128, b);
-                    if (g >= nkb) {
-                        const int vs = gv & 1;
-                        if (!mbar_wait(&v_empty[vs], ((gv >> 1) & 1) ^ 1, abortp)) { ok = false; break; }
-                        mbar_arrive_expect_tx(&v_full[vs], SM::V_BYTES);
+                    if (!mbar_wait(&v_empty[st], ((g >> 1) & 1) ^ 1, abortp)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&v_full[st], SM::V_BYTES);
 #pragma unroll
-                        for (int half = 0; half < 2; ++half)
-                            tma_load_2d(sV + vs * SM::V_BYTES + half * (HD * 128), &tmVt, &v_full[vs],
-                                        j * 128 + half * 64, vt_row);
-                        ++gv;
-                    }
+                    for (int half = 0; half < 2; ++half)
+                        tma_load_2d(sV + st * SM::V_BYTES + half * (HD * 128), &tmVt, &v_full[st], j * 128 + half * 64, vt_row);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            uint32_t gk = 0, gv = 0;
+            uint32_t gs = 0, gv = 0;     // S products and P.V products issued so far
             int it = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
-                const uint32_t o_tmem = tmem_base + O_COL + (it & 1) * 128;
                 auto issue_S = [&](bool last) -> bool {
-                    const int st = gk & 1;
-                    if (!mbar_wait(&k_full[st], (gk >> 1) & 1, abortp)) return false;
-                    if (!mbar_wait(&s_empty[st], ((gk >> 1) & 1) ^ 1, abortp)) return false;
+                    const int st = gs & 1;
+                    if (!mbar_wait(&k_full[st], (gs >> 1) & 1, abortp)) return false;
+                    if (!mbar_wait(&s_empty[st], ((gs >> 1) & 1) ^ 1, abortp)) return false;
                     tc_fence_after();
-                    const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * SM::K_BYTES);
+                    const uint64_t qd = umma_desc_k128(smem_u32(sQ)), kd = umma_desc_k128(smem_u32(sK + st * SM::K_BYTES));
 #pragma unroll
                     for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem_base + st * 128, umma_desc_k128(qa + kb * 16384 + k * 32),
-                                      umma_desc_k128(ka + kb * 16384 + k * 32), IDESC_S, (kb | k) != 0);
+                            umma_bf16(tmem_base + st * 128, qd + kb * 1024 + 2 * k, kd + kb * 1024 + 2 * k, IDESC_S, (kb | k) != 0);
                     umma_commit(&k_empty[st]);
                     umma_commit(&s_full[st]);
                     if (last) umma_commit(&q_empty);          // Q may now be overwritten by the next item's
-                    ++gk;
+                    ++gs;
                     return true;
                 };
                 auto issue_PV = [&](int j) -> bool {
                     const int vs = gv & 1;
                     if (!mbar_wait(&v_full[vs], (gv >> 1) & 1, abortp)) return false;
                     if (!mbar_wait(&p_full, gv & 1, abortp)) return false;
+                    // the first product of an item overwrites the accumulators: the previous item's output step must be done
+                    if (j == 0 && !mbar_wait(&o_empty, (it & 1) ^ 1, abortp)) return false;
                     tc_fence_after();
-                    const uint32_t pa = smem_u32(sP), va = smem_u32(sV + vs * SM::V_BYTES);
+                    const uint64_t pd = umma_desc_k128(smem_u32(sP)), vd = umma_desc_k128(smem_u32(sV + vs * SM::V_BYTES));
+                    // the left 64 keys of the block feed O_left, the right 64 feed O_right
 #pragma unroll
                     for (int half = 0; half < 2; ++half)
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            umma_bf16(o_tmem, umma_desc_k128(pa + half * 16384 + k * 32),
-                                      umma_desc_k128(va + half * (HD * 128) + k * 32), IDESC_O, (j | half | k) != 0);
+                            umma_bf16(tmem_base + O_COL + half * 128, pd + half * 1024 + 2 * k, vd + half * (HD * 8) + 2 * k,
+                                      IDESC_O, (j | k) != 0);
                     umma_commit(&v_empty[vs]);
                     umma_commit(&p_empty);
-                    if (j == nkb - 1) umma_commit(&o_full[it & 1]);
+                    if (j == nkb - 1) umma_commit(&o_full);
                     ++gv;
                     return true;
                 };
                 ok = mbar_wait(&q_full, it & 1, abortp);
-                // this item's O buffer must have been drained by the output step of the item two before
-                ok = ok && mbar_wait(&o_empty[it & 1], ((it >> 1) & 1) ^ 1, abortp);
-                ok = ok && issue_S(false);
-                for (int g = 1; ok && g < 2 * nkb; ++g) {
-                    ok = issue_S(g == 2 * nkb - 1);
-                    if (ok && g - 1 >= nkb) ok = issue_PV(g - 1 - nkb);
+                ok = ok && issue_S(nkb == 1);
+                for (int j = 1; ok && j < nkb; ++j) {
+                    ok = issue_S(j == nkb - 1);
+                    if (ok) ok = issue_PV(j - 1);
                 }
                 if (ok) ok = issue_PV(nkb - 1);
             }
@@ -212,66 +219,103 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
         const int quad = warp & 3, hf = (warp - 2) >> 2;
         const int r = quad * 32 + lane;
         const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);
+        const uint32_t o_mine = lane_base + O_COL + hf * 128;      // this thread's row of ITS accumulator
         const float c = p.scale_log2e;
-        uint32_t gk = 0, gv = 0;
+        uint32_t g = 0;
         int it = 0;
         bool ok = true;
+        // The tensor-memory loads and stores below are warp-wide instructions: the 32 threads of a warp must reach
+        // them together.  So every wait is followed by a vote, and a warp leaves the loops as one.
+        auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+            const bool w = mbar_wait(bar, parity, abortp);
+            return __all_sync(0xffffffffu, w);
+        };
         for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
             int q_blk, h, b;
             decode(item, q_blk, h, b);
-            // ---- pass 1: row maximum of the raw scores ----
-            float m = -INFINITY;
-            for (int j = 0; ok && j < nkb; ++j, ++gk) {
-                const int st = gk & 1;
-                if (!mbar_wait(&s_full[st], (gk >> 1) & 1, abortp)) { ok = false; break; }
+            float mc = -INFINITY, l = 0.f;          // reference maximum (scaled to base-2 exponents) and row sum
+            for (int j = 0; ok && j < nkb; ++j, ++g) {
+                const int st = g & 1;
+                ATTN_T(t0);
+                if (!wait_all(&s_full[st], (g >> 1) & 1)) { ok = false; break; }
+                ATTN_T(t1);
+                ATTN_ACC(0, t0, t1);
                 tc_fence_after();
-#pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    float v[32];
-                    tmem_ld32(lane_base + st * 128 + hf * 64 + ch * 32, v);
-                    tmem_ld_wait();
-                    const int key0 = j * 128 + hf * 64 + ch * 32;
-#pragma unroll
-                    for (int t = 0; t < 32; ++t) m = (key0 + t < L) ? fmaxf(m, v[t]) : m;
-                }
+                float v[64];
+                tmem_ld32(lane_base + st * 128 + hf * 64, v);
+                tmem_ld32(lane_base + st * 128 + hf * 64 + 32, v + 32);
+                tmem_ld_wait_regs(v);
+                tmem_ld_wait_regs(v + 32);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s_empty[st]);
-            }
-            if (!ok) break;
-            // the two halves of a row meet (bounded wait, like every other wait in this kernel)
-            x_max[hf][r] = m;
-            mbar_arrive(&xmax_bar);
-            if (!mbar_wait(&xmax_bar, it & 1, abortp)) { ok = false; break; }
-            m = fmaxf(m, x_max[hf ^ 1][r]);
-            // ---- pass 2: probabilities, P to shared memory, row sum ----
-            const float mc = m * c;
-            float l = 0.f;
-            for (int j = 0; ok && j < nkb; ++j, ++gk, ++gv) {
-                const int st = gk & 1;
-                if (!mbar_wait(&s_full[st], (gk >> 1) & 1, abortp)) { ok = false; break; }
-                tc_fence_after();
+                ATTN_T(t2);
+                ATTN_ACC(1, t1, t2);
+                const int key0 = j * 128 + hf * 64;
+                const bool whole = key0 + 64 <= L;            // every key of this half exists: no per-key bound checks
+                float bm = -INFINITY;
+                if (whole) {
+#pragma unroll
+                    for (int t = 0; t < 64; t += 2) bm = fmaxf(bm, fmaxf(v[t], v[t + 1]));
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 64; ++t) bm = (key0 + t < L) ? fmaxf(bm, v[t]) : bm;
+                }
+                const float bmc = bm * c;
+                const bool raise = bmc > mc + kRaise || (mc == -INFINITY && bm > -INFINITY);
+                const bool shrink = raise && j > 0 && mc > -INFINITY;       // something accumulated against the old reference
+                // where the reference rises, what was accumulated so far shrinks by 2^(old - new); by 1 elsewhere
+                const float f = shrink ? ex2_approx(mc - bmc) : 1.f;
+                if (raise) mc = bmc;
+                l *= f;
                 uint32_t packed[32];
+                if (whole) {                                  // (mc is finite here: the half has keys)
+                    float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    float v[32];
-                    tmem_ld32(lane_base + st * 128 + hf * 64 + ch * 32, v);
-                    tmem_ld_wait();
-                    const int key0 = j * 128 + hf * 64 + ch * 32;
+                    for (int t = 0; t < 32; ++t) {
+                        const float e0 = ex2_approx(fmaf(v[2 * t], c, -mc));
+                        const float e1 = ex2_approx(fmaf(v[2 * t + 1], c, -mc));
+                        l0 += e0;
+                        l1 += e1;
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(e0, e1);
+                        packed[t] = *reinterpret_cast<uint32_t*>(&h2);
+                    }
+                    l += l0 + l1;
+                } else if (mc > -INFINITY) {
 #pragma unroll
-                    for (int t = 0; t < 16; ++t) {
-                        float e0 = (key0 + 2 * t < L) ? ex2_approx(fmaf(v[2 * t], c, -mc)) : 0.f;
-                        float e1 = (key0 + 2 * t + 1 < L) ? ex2_approx(fmaf(v[2 * t + 1], c, -mc)) : 0.f;
+                    for (int t = 0; t < 32; ++t) {
+                        const float e0 = (key0 + 2 * t < L) ? ex2_approx(fmaf(v[2 * t], c, -mc)) : 0.f;
+                        const float e1 = (key0 + 2 * t + 1 < L) ? ex2_approx(fmaf(v[2 * t + 1], c, -mc)) : 0.f;
                         l += e0 + e1;
                         __nv_bfloat162 h2 = __floats2bfloat162_rn(e0, e1);
-                        packed[ch * 16 + t] = *reinterpret_cast<uint32_t*>(&h2);
+                        packed[t] = *reinterpret_cast<uint32_t*>(&h2);
                     }
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 32; ++t) packed[t] = 0u;          // no valid key in this half so far
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&s_empty[st]);
-                // P buffer free once the previous P.V has retired
-                if (!mbar_wait(&p_empty, (gv & 1) ^ 1, abortp)) { ok = false; break; }
+                // the P buffer, and this thread's accumulator row, are free once the previous P.V has retired
+                ATTN_T(t3);
+                ATTN_ACC(2, t2, t3);
+                if (!wait_all(&p_empty, (g & 1) ^ 1)) { ok = false; break; }
+                ATTN_T(t4);
+                ATTN_ACC(3, t3, t4);
+                if (__any_sync(0xffffffffu, shrink)) {
+                    // warp-uniform branch (tensor-memory loads and stores are warp-wide): every thread passes its
+                    // accumulator row through
+                    tc_fence_after();
+#pragma unroll
+                    for (int ch = 0; ch < HD / 32; ++ch) {
+                        float o[32];
+                        tmem_ld32(o_mine + ch * 32, o);
+                        tmem_ld_wait_regs(o);
+#pragma unroll
+                        for (int t = 0; t < 32; ++t) o[t] *= f;
+                        tmem_st32(o_mine + ch * 32, o);
+                    }
+                    tmem_st_wait();
+                    tc_fence_before();
+                }
                 // this thread's 64 keys = sub-tile hf of P, row r: 8 chunks of 16 bytes, 128-byte swizzle
 #pragma unroll
                 for (int cc = 0; cc < 8; ++cc) {
@@ -279,25 +323,41 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
                     *reinterpret_cast<uint4*>(dst) =
                         make_uint4(packed[cc * 4], packed[cc * 4 + 1], packed[cc * 4 + 2], packed[cc * 4 + 3]);
                 }
+                // every thread makes its own stores visible to the tensor core's proxy; one arrival per warp (256 single
+                // arrivals on one barrier cost more than the block's arithmetic)
                 fence_proxy_async_smem();
-                mbar_arrive(&p_full);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full);
+                ATTN_T(t5);
+                ATTN_ACC(4, t4, t5);
+                ATTN_ACC(6, t0, t0 + 1);
             }
             if (!ok) break;
+            // ---- the two halves of a row meet ----
+            ATTN_T(t6);
+            x_max[hf][r] = mc;
             x_sum[hf][r] = l;
-            mbar_arrive(&xsum_bar);
-            if (!mbar_wait(&xsum_bar, it & 1, abortp)) { ok = false; break; }
-            l += x_sum[hf ^ 1][r];
-            // ---- output: this thread's half of the head dimension ----
-            if (!mbar_wait(&o_full[it & 1], (it >> 1) & 1, abortp)) { ok = false; break; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&x_bar);
+            if (!wait_all(&x_bar, it & 1)) { ok = false; break; }
+            const float mo = x_max[hf ^ 1][r], lo = x_sum[hf ^ 1][r];
+            const float m = fmaxf(mc, mo);
+            const float a_me = mc > -INFINITY ? ex2_approx(mc - m) : 0.f;
+            const float a_ot = mo > -INFINITY ? ex2_approx(mo - m) : 0.f;
+            const float inv_l = 1.f / (l * a_me + lo * a_ot);
+            const float w_mine = a_me * inv_l, w_other = a_ot * inv_l;
+            // ---- output: this thread's half of the head dimension, from both accumulators ----
+            if (!wait_all(&o_full, it & 1)) { ok = false; break; }
             tc_fence_after();
             const int q = q_blk * 128 + r;
-            const float inv_l = 1.f / l;
 #pragma unroll
             for (int ch = 0; ch < HD / 64; ++ch) {
-                float v[32];
+                float a[32], bb[32];
                 const int col = hf * (HD / 2) + ch * 32;
-                tmem_ld32(lane_base + O_COL + (it & 1) * 128 + col, v);
-                tmem_ld_wait();
+                tmem_ld32(lane_base + O_COL + hf * 128 + col, a);
+                tmem_ld32(lane_base + O_COL + (hf ^ 1) * 128 + col, bb);
+                tmem_ld_wait_regs(a);
+                tmem_ld_wait_regs(bb);
                 if (q < p.q_cnt) {
                     __nv_bfloat16* dst = p.out + ((size_t)b * p.q_cnt + q) * (size_t)(p.nq * HD) + h * HD + col;
 #pragma unroll
@@ -305,15 +365,19 @@ attention_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmQKV, 
                         uint4 ov;
                         __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
 #pragma unroll
-                        for (int t = 0; t < 4; ++t)
-                            o2[t] = __floats2bfloat162_rn(v[g4 * 8 + 2 * t] * inv_l, v[g4 * 8 + 2 * t + 1] * inv_l);
+                        for (int t = 0; t < 4; ++t) {
+                            const int e = g4 * 8 + 2 * t;
+                            o2[t] = __floats2bfloat162_rn(a[e] * w_mine + bb[e] * w_other, a[e + 1] * w_mine + bb[e + 1] * w_other);
+                        }
                         *reinterpret_cast<uint4*>(dst + g4 * 8) = ov;
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&o_empty[it & 1]);
+            if (lane == 0) mbar_arrive(&o_empty);
+            ATTN_T(t7);
+            ATTN_ACC(5, t6, t7);
         }
     }
 

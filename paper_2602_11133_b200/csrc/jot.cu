@@ -1419,6 +1419,16 @@ int noalloc_scratch_address(float** out) {
 }
 }  // namespace
 
+#ifdef JOT_ATTN_TRACE
+extern "C" int jot_debug_attn_trace(long long* h_out, int n_words, int reset) {
+    if (reset) {
+        static long long zeros[256 * 8] = {};
+        return cudaMemcpyToSymbol(g_attn_trace, zeros, sizeof(zeros)) == cudaSuccess ? 0 : -4;
+    }
+    return cudaMemcpyFromSymbol(h_out, g_attn_trace, (size_t)n_words * 8) == cudaSuccess ? 0 : -4;
+}
+#endif
+
 #ifdef JOT_SLAB_TRACE
 extern "C" int jot_debug_slab_trace(unsigned long long* h_out, int n_words) {
     return cudaMemcpyFromSymbol(h_out, g_slab_trace, (size_t)n_words * 8) == cudaSuccess ? 0 : -4;

@@ -66,6 +66,44 @@ def test_denoise_step_matches_oracle(jot, name, B, P, G, p_mask):
     model.close()
 
 
+@pytest.mark.parametrize("name,B,L", [("tiny", 1, 384), ("hd128", 2, 300), ("gqa", 1, 137)])
+def test_attention_with_scores_that_keep_rising(jot, name, B, L):
+    """Attention keeps a lazy reference maximum per half row and rescales its accumulator in tensor memory when a
+    later key block tops it by more than 2^8.  Ordinary random-init weights never get there, so this model has
+    query / key projections 50 times larger: the scores spread over hundreds, every row raises its reference
+    several times, and the softmax is nearly one-hot.  Hidden states after one layer against the oracle."""
+    g = GEOMS[name]
+    w_cpu = inputs.model_weights(g, seed=0, n_layers=1)
+    qk_rows = (g.n_q_heads + g.n_kv_heads) * g.head_dim
+    big = inputs.normal(11, "big_qk", (qk_rows, g.d_model), 1.0)
+    w_cpu["layers"][0]["wqkv"] = torch.cat([big, w_cpu["layers"][0]["wqkv"][qk_rows:]]).contiguous()
+    w_gpu = inputs.weights_to(w_cpu, "cuda")
+    tokens = inputs.partially_masked_canvas(2, B, L // 3, L - L // 3, g.vocab, g.mask_id, 0.5)
+    model = jot.Model(g, w_gpu, B, L)
+    st = model.denoise_step(tokens.cuda(), L // 3, L)
+    torch.cuda.synchronize()
+    rows = [(b, i) for b in range(B) for i in range(L // 3, L) if int(tokens[b, i]) == g.mask_id]
+    # how far the scores rise from one key block of 128 to a later one (oracle side, first head)
+    lw = w_cpu["layers"][0]
+    a = mo._r(mo.rmsnorm(w_cpu["embed"][tokens.long()].double(), lw["attn_norm"], g.rms_eps), True)
+    qkv = mo._r(a @ lw["wqkv"].double().T, True)
+    q = mo.rope(qkv[..., :g.head_dim].reshape(B, L, 1, g.head_dim), g.rope_theta)
+    k = mo.rope(qkv[..., g.n_q_heads * g.head_dim: g.n_q_heads * g.head_dim + g.head_dim].reshape(B, L, 1, g.head_dim), g.rope_theta)
+    s = torch.einsum("blhd,bmhd->blm", q, k) / math.sqrt(g.head_dim) * math.log2(math.e)
+    if L > 128:
+        rise = (s[:, :, 128:].max(dim=-1).values - s[:, :, :128].max(dim=-1).values)
+        assert int((rise > 8).sum()) > (L // 4 if L >= 256 else 0), "the case must make the reference maximum move"
+    logits = mo.logits(g, w_cpu, tokens, rows=rows)
+    want = oracle_stats_for_rows(logits, g.mask_id)
+    flat = torch.tensor([b * L + i for b, i in rows])
+    pick = lambda t: t.cpu().view(-1)[flat].numpy()
+    n, near = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), want, rel=REL_TOL,
+                            gap_from_tolerance=True)
+    print(f"{name} with rising scores: {n} rows checked, max |top1 err| "
+          f"{max(abs(x - w.m1) for x, w in zip(pick(st.top1), want)):.2e}")
+    model.close()
+
+
 def oracle_trajectory(g, w_cpu, prompt_row, G, T, params, block_len, bump=None):
     def logits_fn(x, rows):
         t = torch.tensor([x], dtype=torch.int32)
@@ -106,7 +144,9 @@ def test_tiny_generation_teacher_forced_and_free_running(jot, params, block_len,
         assert excused <= 2
         assert tr.steps_used < T          # the bump makes positions exit early
     else:
-        assert excused <= 0.75 * len(tr.canvases)      # measured: 38-40 of 63 picks among near-equal confidences
+        # positions are counted, two per swapped pick: at most half of the steps may pick another of the near-equal
+        # candidates (measured: 19-28 of 63 steps, depending on the rounding pattern of the attention kernel)
+        assert excused <= len(tr.canvases)
 
     out, used, passes = model.generate(prompt.cuda(), G, T, jp, block_len, **d_bump)
     got = out.cpu()[0].tolist()
