@@ -382,9 +382,12 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
-    // everything above is on-chip; from here on global memory written by earlier kernels is read
+    // everything above is on-chip; from here on global memory written by earlier kernels is read.  The LM-head
+    // schedule depends on a device word the preceding kernel wrote, so that kernel waits here; the others let
+    // every role wait for itself, and the producer requests its first W tiles BEFORE it waits (the weights are
+    // nobody's output): the pipeline fill overlaps the predecessor's tail.
     grid_launch_dependents();
-    grid_dependency_wait();
+    if (EPI == EPI_STATS) grid_dependency_wait();
 
 
     // ---- tile schedule (identical in every role) ----
@@ -442,22 +445,42 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         uint32_t phase = 0;
         int m_blk, n_blk;
         bool ok = true;
+        auto load_w = [&](int st, int kb, int nb) {
+            uint8_t* sB = smem + st * SM::STAGE_BYTES + SM::A_BYTES;
+            mbar_arrive_expect_tx(&full_bar[st], SM::STAGE_BYTES);
+            if (EPI == EPI_SWIGLU) {
+                // gate rows, then the matching up rows: two boxes of BN/2 rows each
+                tma_load_2d(sB, &tmB, &full_bar[st], kb * kBK, nb * (BN / 2));
+                tma_load_2d(sB + SM::B_BYTES / 2, &tmB, &full_bar[st], kb * kBK, p.N / 2 + nb * (BN / 2));
+            } else {
+                tma_load_2d(sB, &tmB, &full_bar[st], kb * kBK, nb * BN);
+            }
+        };
+        // the first tile's first W tiles go out before the wait on the preceding kernel, its A tiles after
+        int n_pre = 0;
+        if (EPI != EPI_STATS) {
+            if (tile_at(0, m_blk, n_blk)) {
+                n_pre = min(STAGES, kb1 - kb0);
+                if (elected)
+                    for (int i = 0; i < n_pre; ++i) load_w(i, kb0 + i, n_blk);
+            }
+            __syncwarp();
+            grid_dependency_wait();
+            if (elected)
+                for (int i = 0; i < n_pre; ++i)
+                    tma_load_2d(smem + i * SM::STAGE_BYTES, &tmA, &full_bar[i], (kb0 + i) * kBK, m_blk * kBM);
+            __syncwarp();
+        }
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             for (int kb = kb0; kb < kb1; ++kb) {
+                if (it == 0 && kb - kb0 < n_pre) {            // already requested above
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    continue;
+                }
                 if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
-                uint8_t* sA = smem + stage * SM::STAGE_BYTES;
-                uint8_t* sB = sA + SM::A_BYTES;
                 if (elected) {
-                    mbar_arrive_expect_tx(&full_bar[stage], SM::STAGE_BYTES);
-                    tma_load_2d(sA, &tmA, &full_bar[stage], kb * kBK, m_blk * kBM);
-                    if (EPI == EPI_SWIGLU) {
-                        // gate rows, then the matching up rows: two boxes of BN/2 rows each
-                        tma_load_2d(sB, &tmB, &full_bar[stage], kb * kBK, n_blk * (BN / 2));
-                        tma_load_2d(sB + SM::B_BYTES / 2, &tmB, &full_bar[stage], kb * kBK,
-                                    p.N / 2 + n_blk * (BN / 2));
-                    } else {
-                        tma_load_2d(sB, &tmB, &full_bar[stage], kb * kBK, n_blk * BN);
-                    }
+                    load_w(stage, kb, n_blk);
+                    tma_load_2d(smem + stage * SM::STAGE_BYTES, &tmA, &full_bar[stage], kb * kBK, m_blk * kBM);
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -503,6 +526,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         __syncwarp();
     } else {
         // ================= epilogue (warps 2..5) =================
+        if (EPI != EPI_STATS) grid_dependency_wait();     // residual, rotary table: written or read after earlier kernels
         const int quad = warp & 3;                        // TMEM lanes [32*quad, 32*quad+32)
         const int row_in_tile = quad * 32 + lane;
         const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);

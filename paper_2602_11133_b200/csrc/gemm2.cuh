@@ -73,8 +73,10 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abortp = &abort_flag;
+    // as in the one-CTA kernel: the LM-head schedule needs a device word of the preceding kernel; the other
+    // epilogues let each role wait for itself, the producer after it has requested its first W tiles
     grid_launch_dependents();
-    grid_dependency_wait();
+    if (EPI == EPI_STATS) grid_dependency_wait();
 
     // ---- schedule: pair tiles (two row blocks x one 256-wide column block), identical in every role ----
     const int num_m = (p.M + kBM - 1) / kBM, num_pm = (num_m + 1) / 2;
@@ -121,11 +123,36 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         uint32_t phase = 0;
         int m_blk, n_blk;
         bool ok = true;
+        // this CTA's half of the W tile: SwiGLU pairs 128 gate rows (leader) with the matching 128 up rows
+        auto w_row_of = [&](int nb) {
+            return (EPI == EPI_SWIGLU) ? (rank == 0 ? nb * kBM : p.N / 2 + nb * kBM) : nb * BN + rank * kBM;
+        };
+        // the first tile's first W tiles go out before the wait on the preceding kernel, its A tiles after
+        int n_pre = 0;
+        if (EPI != EPI_STATS) {
+            if (tile_at(0, m_blk, n_blk)) {
+                n_pre = min(STAGES, num_kb);
+                if (elected)
+                    for (int i = 0; i < n_pre; ++i) {
+                        if (leader) mbar_arrive_expect_tx(&full_bar[i], 2 * kPairStageBytes);
+                        tma_load_2d_pair(smem + i * kPairStageBytes + HALF_BYTES, &tmB, mapa_u32(&full_bar[i], 0), i * kBK,
+                                         w_row_of(n_blk));
+                    }
+            }
+            __syncwarp();
+            grid_dependency_wait();
+            if (elected)
+                for (int i = 0; i < n_pre; ++i)
+                    tma_load_2d_pair(smem + i * kPairStageBytes, &tmA, mapa_u32(&full_bar[i], 0), i * kBK, m_blk * kBM);
+            __syncwarp();
+        }
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
-            // this CTA's half of the W tile: SwiGLU pairs 128 gate rows (leader) with the matching 128 up rows
-            const int w_row = (EPI == EPI_SWIGLU) ? (rank == 0 ? n_blk * kBM : p.N / 2 + n_blk * kBM)
-                                                  : n_blk * BN + rank * kBM;
+            const int w_row = w_row_of(n_blk);
             for (int kb = 0; kb < num_kb; ++kb) {
+                if (it == 0 && kb < n_pre) {                  // already requested above
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    continue;
+                }
                 if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) { ok = false; break; }
                 uint8_t* sA = smem + stage * kPairStageBytes;
                 uint8_t* sB = sA + HALF_BYTES;
@@ -182,6 +209,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         __syncwarp();
     } else {
         // ================= epilogue (warps 2..5, both CTAs) =================
+        if (EPI != EPI_STATS) grid_dependency_wait();
         const int quad = warp & 3;
         const int row_in_tile = quad * 32 + lane;
         const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);

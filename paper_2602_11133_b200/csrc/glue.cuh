@@ -126,25 +126,31 @@ __global__ void __launch_bounds__(512) splitk_reduce_norm_kernel(const float* __
                                                                   int N, const __nv_bfloat16* __restrict__ gain,
                                                                   __nv_bfloat16* __restrict__ out, float eps) {
     grid_launch_dependents();
-    grid_dependency_wait();
     __shared__ float scratch[33];
     const int row = blockIdx.x, nvec = N / 8;
     const size_t total = (size_t)M * N, base = (size_t)row * N;
     constexpr int MAXV = 2, MAXS = 4;
     float4 pa[MAXV][MAXS][2];
     uint4 rv[MAXV], gv[MAXV];
+    // The gain is a weight, nobody's output: it is requested before the wait on the preceding kernel.  (The
+    // residual is not: with programmatic launches the kernel before the preceding one may still be writing it.)
+#pragma unroll
+    for (int t = 0; t < MAXV; ++t) {
+        const int i = threadIdx.x + t * blockDim.x;
+        if (i < nvec) gv[t] = *reinterpret_cast<const uint4*>(gain + i * 8);
+    }
+    grid_dependency_wait();
 #pragma unroll
     for (int t = 0; t < MAXV; ++t) {
         const int i = threadIdx.x + t * blockDim.x;
         if (i < nvec) {
+            rv[t] = residual ? *reinterpret_cast<const uint4*>(residual + base + i * 8) : make_uint4(0, 0, 0, 0);
 #pragma unroll
             for (int s = 0; s < MAXS; ++s)
                 if (s < split) {
                     pa[t][s][0] = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8);
                     pa[t][s][1] = *reinterpret_cast<const float4*>(partial + s * total + base + i * 8 + 4);
                 }
-            rv[t] = residual ? *reinterpret_cast<const uint4*>(residual + base + i * 8) : make_uint4(0, 0, 0, 0);
-            gv[t] = *reinterpret_cast<const uint4*>(gain + i * 8);
         }
     }
     uint4 hbuf[MAXV];
