@@ -25,7 +25,7 @@ def oracle_stats_for_rows(logits_rows: torch.Tensor, mask_id) -> List[jo.RowStat
 
 
 def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowStats], rel=REL_TOL,
-                  gap_from_tolerance=False):
+                  gap_from_tolerance=False, gap_from_error=False):
     """Returns (n_checked, n_near_tie).  Raises AssertionError on a real mismatch.
 
     The argmax must agree unless the oracle's top-2 gap is below GAP_TOL.  With gap_from_tolerance (deep
@@ -34,9 +34,13 @@ def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowS
     2*rel*scale.  Exempt rows are counted, and their argmax must still be the oracle's runner-up region:
     the GPU's top-1 logit has to be within tolerance of the oracle's."""
     near = strict = differ = 0
+    # gap_from_error: the exemption is what THIS comparison's own logit error allows: two logits that are each off by
+    # at most e can only swap when they are closer than 2 e (e = the largest top-1 / runner-up error over the rows)
+    e_max = max([max(abs(got_top1[r] - st.m1), abs(got_top2[r] - st.m2)) for r, st in enumerate(want)] or [0.0])
     for r, st in enumerate(want):
         scale = max(abs(st.m1), abs(st.m2), 1.0)
-        gap_tol = max(GAP_TOL, 2 * rel * scale) if gap_from_tolerance else GAP_TOL
+        gap_tol = max(GAP_TOL, 2 * rel * scale) if gap_from_tolerance else (
+            max(GAP_TOL, 2 * float(e_max)) if gap_from_error else GAP_TOL)
         assert abs(got_top1[r] - st.m1) <= rel * scale, (r, got_top1[r], st.m1)
         assert abs(got_top2[r] - st.m2) <= rel * scale, (r, got_top2[r], st.m2)
         # log-sum-exp agrees to the logit tolerance  <=> S agrees to a relative factor
@@ -48,7 +52,7 @@ def compare_stats(got_top1, got_top2, got_sumexp, got_argmax, want: List[jo.RowS
         else:
             assert int(got_argmax[r]) == st.i1, (r, int(got_argmax[r]), st.i1, st.m1 - st.m2)
     LAST_COMPARE.update(rows=len(want), inside_margin=near, inside_strict_margin=strict, argmax_differs=differ)
-    if gap_from_tolerance:
+    if gap_from_tolerance or gap_from_error:
         print(f"compare_stats: {len(want)} rows; top-2 gap inside the widened margin: {near} "
               f"(of which inside the strict {GAP_TOL:g} margin: {strict}); argmax actually different: {differ}")
     return len(want), near

@@ -29,6 +29,21 @@ def jot():
 ])
 @pytest.mark.parametrize("with_res", [False, True])
 def test_gemm_matches_float64_definition(jot, M, N, K, with_res):
+    check_gemm(jot, M, N, K, with_res)
+
+
+# canvases of at most 512 rows without scratch run the slab kernel: one or two accumulators, K cut over the CTA pairs
+# of a cluster (2, 3 or 4 ranges, reduce-scatter through distributed shared memory) when there are few slabs
+@pytest.mark.parametrize("M,N,K", [
+    (1, 256, 64), (31, 136, 72), (255, 520, 1096), (257, 264, 200), (512, 1024, 512), (448, 4096, 1024),
+    (96, 512, 4096), (200, 2048, 2048), (384, 1032, 12288), (320, 256, 8192),
+])
+@pytest.mark.parametrize("with_res", [False, True])
+def test_gemm_small_canvas_shapes(jot, M, N, K, with_res):
+    check_gemm(jot, M, N, K, with_res)
+
+
+def check_gemm(jot, M, N, K, with_res):
     a = inputs.normal(1, "a", (M, K), 1.0).cuda()
     w = inputs.normal(1, "w", (N, K), 0.05).cuda()
     res = inputs.normal(1, "r", (M, N), 1.0).cuda() if with_res else None

@@ -37,6 +37,11 @@ def masked_canvas(seed, B, P, G, g, p_mask):
     ("tiny", 2, 60, 140, 0.5),         # L = 200: two key blocks with a ragged tail, two sequences
     ("gqa", 3, 17, 120, 0.7),          # L = 137
     ("hd128", 2, 128, 256, 0.5),       # L = 384: three key blocks
+    # canvases of at most 256 rows run the slab projection kernel (weight rows as the MMA's M side)
+    ("gqa", 1, 17, 120, 0.7),          # 137 rows: one accumulator of 160 columns, ragged everything
+    ("hd128", 1, 64, 192, 0.5),        # 256 rows: the largest canvas on that path, one head per CTA
+    ("tiny", 2, 30, 70, 0.6),          # 200 rows, two sequences in one token tile, two heads per CTA
+    ("tiny", 1, 8, 24, 1.0),           # 32 rows: the smallest accumulator
 ])
 def test_denoise_step_matches_oracle(jot, name, B, P, G, p_mask):
     g = GEOMS[name]
@@ -52,10 +57,16 @@ def test_denoise_step_matches_oracle(jot, name, B, P, G, p_mask):
     want = oracle_stats_for_rows(logits, g.mask_id)
     flat = torch.tensor([b * L + i for b, i in rows])
     pick = lambda t: t.cpu().view(-1)[flat].numpy()
-    n, near = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), want, rel=REL_TOL)
-    print(f"{name}: {n} rows, {near} with top-2 gap < {GAP_TOL}, max |top1 err| "
+    # a model without the planted bump has many near-equal logits: the argmax must agree wherever the two largest are
+    # further apart than twice the largest logit error of this very comparison (never less than the strict 1e-3)
+    n, near = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), want, rel=REL_TOL,
+                            gap_from_error=True)
+    print(f"{name}: {n} rows, {near} with a top-2 gap inside that margin, max |top1 err| "
           f"{max(abs(a - s.m1) for a, s in zip(pick(st.top1), want)):.2e}")
-    assert near <= max(2, n // 20)
+    import helpers
+    # outside the margin the argmax was required to be equal; inside it a flip is legitimate, but a broken argmax
+    # would flip most of those rows, not a fraction
+    assert helpers.LAST_COMPARE["argmax_differs"] <= max(2, helpers.LAST_COMPARE["inside_margin"] // 4)
     # the same against the oracle without any bf16 rounding of activations: the plain float64 network
     plain = oracle_stats_for_rows(mo.logits(g, w_cpu, tokens, rows=rows, round_activations=False), g.mask_id)
     n2, near2 = compare_stats(pick(st.top1), pick(st.top2), pick(st.sumexp), pick(st.argmax), plain, rel=REL_TOL,
