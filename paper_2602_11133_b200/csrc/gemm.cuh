@@ -7,7 +7,8 @@
 //                      at a time and applies one of three epilogues:
 //        EPI_STORE   bf16(acc [+ residual])                                  -> C[M, N]
 //        EPI_SWIGLU  bf16(silu(gate) * up), gate/up from the two halves of W -> C[M, N/2]
-//        EPI_STATS   online (max, argmax, runner-up, sum-exp) per row over a range of vocabulary tiles;
+//        EPI_STATS   online (max, argmax, runner-up, sum-exp) per row over a range of vocabulary tiles
+//                    (EPI_STATS_DRAW: plus one Gumbel-max draw per row);
 //                    the logits are never written (LM head of the denoising step)
 //        EPI_QKV     QKV projection: bf16(acc), then rotary embedding on the Q and K heads (rotate-half,
 //                    table lookup by canvas position) written to C, and the V heads written transposed
@@ -20,7 +21,10 @@
 
 namespace jot {
 
-enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2, EPI_PARTIAL = 3, EPI_QKV = 4 };
+enum { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_STATS = 2, EPI_PARTIAL = 3, EPI_QKV = 4, EPI_STATS_DRAW = 5 };
+// EPI_STATS_DRAW is EPI_STATS plus the Gumbel-max draw of sampling-based finalisation: an instance of its own, so
+// that the argmax-only head does not carry the draw's registers.
+__host__ __device__ constexpr bool is_stats(int epi) { return epi == EPI_STATS || epi == EPI_STATS_DRAW; }
 
 // Pipeline depth (shared-memory stages of one A tile + one W tile); both fill ~192 KB.
 #ifndef JOT_GEMM_STAGES_256
@@ -303,7 +307,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t t_ac
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = (col0 + j < hi_col && col0 + j >= p.col_lo) ? v[j] : -INFINITY;
             }
-            if (p.inv_temperature > 0.f) {
+            if (EPI == EPI_STATS_DRAW) {
                 // Gumbel-max: argmax_v (l_v / T - ln(-ln u_v)), u_v from 23 bits of the row's counter stream
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
@@ -387,7 +391,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     // every role wait for itself, and the producer requests its first W tiles BEFORE it waits (the weights are
     // nobody's output): the pipeline fill overlaps the predecessor's tail.
     grid_launch_dependents();
-    if (EPI == EPI_STATS) grid_dependency_wait();
+    if (is_stats(EPI)) grid_dependency_wait();
 
 
     // ---- tile schedule (identical in every role) ----
@@ -400,10 +404,10 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     int total_tiles = num_m * num_n * split;
     int chunk = 0;
     // EPI_STATS: only the tiles that touch the vocabulary slice are visited
-    const int stats_hi = (EPI == EPI_STATS && p.col_hi > 0) ? p.col_hi : p.N;
-    const int tile_lo = (EPI == EPI_STATS) ? p.col_lo / BN : 0;
-    const int num_nt = (EPI == EPI_STATS) ? (stats_hi + BN - 1) / BN - tile_lo : num_n;
-    if (EPI == EPI_STATS) {
+    const int stats_hi = (is_stats(EPI) && p.col_hi > 0) ? p.col_hi : p.N;
+    const int tile_lo = (is_stats(EPI)) ? p.col_lo / BN : 0;
+    const int num_nt = (is_stats(EPI)) ? (stats_hi + BN - 1) / BN - tile_lo : num_n;
+    if (is_stats(EPI)) {
         int R = *p.d_R, n_rb, n_ch;
         stats_partition(R, gridDim.x, num_nt, &n_rb, &n_ch);
         chunk = n_rb > 0 ? blockIdx.x / n_rb : 0;
@@ -419,7 +423,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
     }
     int kb0 = 0, kb1 = num_kb, ks = 0;            // K-block range of the current work item
     auto tile_at = [&](int it, int& m_blk, int& n_blk) -> bool {
-        if (EPI == EPI_STATS) {
+        if (is_stats(EPI)) {
             if (it >= total_tiles) return false;
             m_blk = m_blk0;
             n_blk = n_first + it;
@@ -458,7 +462,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         };
         // the first tile's first W tiles go out before the wait on the preceding kernel, its A tiles after
         int n_pre = 0;
-        if (EPI != EPI_STATS) {
+        if (!is_stats(EPI)) {
             if (tile_at(0, m_blk, n_blk)) {
                 n_pre = min(STAGES, kb1 - kb0);
                 if (elected)
@@ -526,7 +530,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         __syncwarp();
     } else {
         // ================= epilogue (warps 2..5) =================
-        if (EPI != EPI_STATS) grid_dependency_wait();     // residual, rotary table: written or read after earlier kernels
+        if (!is_stats(EPI)) grid_dependency_wait();     // residual, rotary table: written or read after earlier kernels
         const int quad = warp & 3;                        // TMEM lanes [32*quad, 32*quad+32)
         const int row_in_tile = quad * 32 + lane;
         const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);
@@ -534,7 +538,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
         uint32_t acc_phase = 0;
         int m_blk, n_blk;
         StatsRow st;
-        if (EPI == EPI_STATS && total_tiles > 0) stats_row_init(p, m_blk0 * kBM + row_in_tile, st);
+        if (is_stats(EPI) && total_tiles > 0) stats_row_init(p, m_blk0 * kBM + row_in_tile, st);
         bool ok = true;
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
@@ -547,10 +551,10 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const _
             if (lane == 0) mbar_arrive(&acc_empty[acc]);
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
-        if (EPI == EPI_STATS && ok && total_tiles > 0) {
+        if (is_stats(EPI) && ok && total_tiles > 0) {
             const size_t slot = (size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile;
             p.partials[slot] = make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
-            if (p.inv_temperature > 0.f) p.partials2[slot] = make_float2(st.best, __int_as_float(st.best_i));
+            if (EPI == EPI_STATS_DRAW) p.partials2[slot] = make_float2(st.best, __int_as_float(st.best_i));
         }
     }
 

@@ -76,7 +76,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
     // as in the one-CTA kernel: the LM-head schedule needs a device word of the preceding kernel; the other
     // epilogues let each role wait for itself, the producer after it has requested its first W tiles
     grid_launch_dependents();
-    if (EPI == EPI_STATS) grid_dependency_wait();
+    if (is_stats(EPI)) grid_dependency_wait();
 
     // ---- schedule: pair tiles (two row blocks x one 256-wide column block), identical in every role ----
     const int num_m = (p.M + kBM - 1) / kBM, num_pm = (num_m + 1) / 2;
@@ -86,7 +86,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
     int total_tiles = num_pm * num_n;
     int m_blk0 = 0, n_first = 0, chunk = 0;
     bool stats_row_block_valid = false;
-    if (EPI == EPI_STATS) {
+    if (is_stats(EPI)) {
         // only the tiles that touch the vocabulary slice [col_lo, col_hi) are visited
         const int stats_hi = p.col_hi > 0 ? p.col_hi : p.N;
         const int tile_lo = p.col_lo / BN, num_nt = (stats_hi + BN - 1) / BN - tile_lo;
@@ -103,7 +103,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         }
     }
     auto tile_at = [&](int it, int& m_blk, int& n_blk) -> bool {
-        if (EPI == EPI_STATS) {
+        if (is_stats(EPI)) {
             if (it >= total_tiles) return false;
             m_blk = m_blk0;
             n_blk = n_first + it;
@@ -129,7 +129,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         };
         // the first tile's first W tiles go out before the wait on the preceding kernel, its A tiles after
         int n_pre = 0;
-        if (EPI != EPI_STATS) {
+        if (!is_stats(EPI)) {
             if (tile_at(0, m_blk, n_blk)) {
                 n_pre = min(STAGES, num_kb);
                 if (elected)
@@ -209,7 +209,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         __syncwarp();
     } else {
         // ================= epilogue (warps 2..5, both CTAs) =================
-        if (EPI != EPI_STATS) grid_dependency_wait();
+        if (!is_stats(EPI)) grid_dependency_wait();
         const int quad = warp & 3;
         const int row_in_tile = quad * 32 + lane;
         const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);
@@ -217,7 +217,7 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
         uint32_t acc_phase = 0;
         int m_blk, n_blk;
         StatsRow st;
-        if (EPI == EPI_STATS && total_tiles > 0) stats_row_init(p, m_blk0 * kBM + row_in_tile, st);
+        if (is_stats(EPI) && total_tiles > 0) stats_row_init(p, m_blk0 * kBM + row_in_tile, st);
         bool ok = true;
         for (int it = 0; ok && tile_at(it, m_blk, n_blk); ++it) {
             if (!mbar_wait(&acc_full[acc], acc_phase, abortp)) { ok = false; break; }
@@ -229,10 +229,10 @@ gemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, co
             if (lane == 0) mbar_arrive_cluster(mapa_u32(&acc_empty[acc], 0));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
-        if (EPI == EPI_STATS && ok && total_tiles > 0 && stats_row_block_valid) {
+        if (is_stats(EPI) && ok && total_tiles > 0 && stats_row_block_valid) {
             const size_t slot = (size_t)chunk * p.R_pad + m_blk0 * kBM + row_in_tile;
             p.partials[slot] = make_float4(st.m1, __int_as_float(st.i1), st.m2, st.S);
-            if (p.inv_temperature > 0.f) p.partials2[slot] = make_float2(st.best, __int_as_float(st.best_i));
+            if (EPI == EPI_STATS_DRAW) p.partials2[slot] = make_float2(st.best, __int_as_float(st.best_i));
         }
     }
 

@@ -700,12 +700,15 @@ int lm_head_from_hsel(jot_model* m, int exclude_mask, const int32_t* bump_id, co
         ProfScope ps(m, JOT_PROF_LM_HEAD, st);
         if (mode == 0) {
             bn = 128;
-            JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+            if (sampling) JOT_TRY((launch_gemm_t<128, EPI_STATS_DRAW>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+            else JOT_TRY((launch_gemm_t<128, EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
         } else if (mode == 1) {
-            JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
+            if (sampling) JOT_TRY((launch_gemm_t<256, EPI_STATS_DRAW>(p, m->tm_hsel, m->wlm.m256, grid, st)));
+            else JOT_TRY((launch_gemm_t<256, EPI_STATS>(p, m->tm_hsel, m->wlm.m256, grid, st)));
         } else {
             grid &= ~1;
-            JOT_TRY((launch_pair_t<EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+            if (sampling) JOT_TRY((launch_pair_t<EPI_STATS_DRAW>(p, m->tm_hsel, m->wlm.m128, grid, st)));
+            else JOT_TRY((launch_pair_t<EPI_STATS>(p, m->tm_hsel, m->wlm.m128, grid, st)));
         }
     }
     const int n_vt = ((v_hi > 0 ? v_hi : c.vocab) + bn - 1) / bn - v_lo / bn;     // tiles that touch the slice
