@@ -67,7 +67,7 @@ __host__ __device__ inline SlabGeom slab_geom(int M, int split) {
     g.recv_bytes = (split - 1) * g.cpo * 32 * 512;                // [source][token][128 features] fp32
     const int epi_bytes = g.recv_bytes + 4 * 32 * 512;            // + two fp32 chunk buffers per warp group
     int stages = (kSlabMaxSmem - 2048) / g.stage_bytes;
-    if (stages > 8) stages = 8;
+    if (stages > 12) stages = 12;      // few tokens: small stages, and the weight stream wants many bytes in flight
     g.stages = stages;
     const int pipe = stages * g.stage_bytes;
     g.smem_bytes = (pipe > epi_bytes ? pipe : epi_bytes) + 1024;
@@ -89,7 +89,7 @@ template <int EPI>
 __global__ void __launch_bounds__(kSlabThreads, 1)
 gemm_slab_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                  const __grid_constant__ CUtensorMap tmX1) {
-    constexpr int MAX_STAGES = 8;
+    constexpr int MAX_STAGES = 12;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], acc_full;
