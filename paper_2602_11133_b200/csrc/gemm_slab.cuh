@@ -38,6 +38,10 @@ constexpr int kSlabMaxTokens = 512;        // two accumulators of 256 fp32 colum
 #define JOT_SLAB_PREFER_TOKENS 256
 #endif
 constexpr int kSlabPreferTokens = JOT_SLAB_PREFER_TOKENS;   // measured: up to here this kernel beats the token-major tiles
+#ifndef JOT_SLAB_GATEUP_TOKENS
+#define JOT_SLAB_GATEUP_TOKENS JOT_SLAB_PREFER_TOKENS
+#endif
+constexpr int kSlabGateUpTokens = JOT_SLAB_GATEUP_TOKENS;   // the same switch for the gate/up projection alone
 constexpr int kSlabMaxSmem = 226 * 1024;   // dynamic part; the static barriers take the rest of the 227 KB
 enum { SLAB_STORE = 0, SLAB_SWIGLU = 1, SLAB_QKV = 2 };
 

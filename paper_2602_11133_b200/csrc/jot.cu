@@ -409,7 +409,7 @@ struct jot_model {
     // A-operand maps of the projections for a pass over M rows (rows past M read as zero without memory
     // traffic): one set for the whole canvas, one for the rows of a block
     // (x*: the same buffers as the token operand of the slab kernel, boxes of half an accumulator's tokens)
-    struct ActMaps { int M = -1; bool slab = false; CUtensorMap a, attn, act; SlabMaps xa, xattn, xact; };
+    struct ActMaps { int M = -1; bool slab = false, slab_gate_up = false; CUtensorMap a, attn, act; SlabMaps xa, xattn, xact; };
     ActMaps maps_full, maps_span;
     // block-wise KV cache (caller's memory, optional): per layer the rotated Q/K rows and V^T of the whole canvas
     uint8_t* kv_base = nullptr;
@@ -538,7 +538,8 @@ int encode_act_maps(jot_model* m, jot_model::ActMaps* am, int M) {
     JOT_TRY(make_map_2d(m->di, &am->attn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim, 128));
     JOT_TRY(make_map_2d(m->di, &am->act, m->act, M, c.d_ff, c.d_ff, 128));
     am->slab = M <= kSlabPreferTokens;
-    if (am->slab) {
+    am->slab_gate_up = M > 128 && M <= kSlabGateUpTokens;
+    if (am->slab || am->slab_gate_up) {
         JOT_TRY(make_slab_maps(m->di, &am->xa, m->a, M, c.d_model, c.d_model));
         JOT_TRY(make_slab_maps(m->di, &am->xattn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim));
         JOT_TRY(make_slab_maps(m->di, &am->xact, m->act, M, c.d_ff, c.d_ff));
@@ -649,7 +650,7 @@ int forward_body(jot_model* m, const int32_t* d_tokens, int B, int L, cudaStream
             // (up to 128 rows the token-major tiles stream the gate/up weights faster than the slab kernel's two
             // launches do: measured 39-43 us against 42-47)
             JOT_TRY(run_gemm(m->di, am.a, m->wgu[l], EPI_SWIGLU, p, st, nullptr, 0, nullptr,
-                             am.slab && M > 128 ? &am.xa : nullptr));
+                             am.slab_gate_up ? &am.xa : nullptr));
         }
         p = GemmParams{};
         p.M = M; p.N = d; p.K = c.d_ff; p.C = m->h; p.residual = m->h; p.ldc = d; p.status = status;
