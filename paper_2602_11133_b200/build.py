@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libjot.so")
 SOURCES = ["jot.cu"]
-HEADERS = ["ptx.cuh", "pdl.cuh", "gemm.cuh", "gemm2.cuh", "attention.cuh", "glue.cuh", "accept.cuh"]
+HEADERS = ["ptx.cuh", "pdl.cuh", "gemm.cuh", "gemm2.cuh", "gemm_slab.cuh", "attention.cuh", "glue.cuh", "accept.cuh"]
 
 
 def _nvcc() -> str:
