@@ -1429,7 +1429,7 @@ int noalloc_scratch_address(float** out) {
 #ifdef JOT_ATTN_TRACE
 extern "C" int jot_debug_attn_trace(long long* h_out, int n_words, int reset) {
     if (reset) {
-        static long long zeros[256 * 8] = {};
+        static long long zeros[256 * 16] = {};
         return cudaMemcpyToSymbol(g_attn_trace, zeros, sizeof(zeros)) == cudaSuccess ? 0 : -4;
     }
     return cudaMemcpyFromSymbol(h_out, g_attn_trace, (size_t)n_words * 8) == cudaSuccess ? 0 : -4;
