@@ -198,3 +198,32 @@ def test_dream_shape_generation_with_a_sweep_setting(jot):
     if excused == 0:
         assert man == tr.x and man_used == tr.steps_used
     model.close()
+
+
+@pytest.mark.parametrize("name,B,L", [("dream", 8, 512), ("dream", 8, 256), ("dream", 3, 512), ("llada", 16, 704)])
+def test_copies_of_one_sequence_get_identical_statistics(jot, name, B, L):
+    """Sequences are independent, so B copies of one canvas must come out bit for bit alike, run after run.  With
+    several work items per attention CTA (896 / 448 / 336 / 3072 items on 148 CTAs here) any hand-over between
+    items that goes wrong shows up as a copy that differs; it needs no oracle and covers every row of every copy."""
+    g = inputs.DREAM_7B if name == "dream" else inputs.LLADA_8B
+    P = L // 2
+    w_gpu = inputs.model_weights(g, seed=0, device="cuda", n_layers=1)
+    model = jot.Model(g, w_gpu, B, L)
+    one = inputs.partially_masked_canvas(5, 1, P, L - P, g.vocab, g.mask_id, 0.5, device="cuda")
+    tokens = one.repeat(B, 1).contiguous()
+    first = None
+    for rep in range(3):
+        st = model.denoise_step(tokens, P, L)
+        torch.cuda.synchronize()
+        active = tokens[0] == g.mask_id
+        active[:P] = False
+        assert int(active.sum()) > 20
+        got = [t[:, active].clone() for t in (st.top1, st.top2, st.sumexp, st.argmax)]
+        assert all(torch.isfinite(t).all() for t in got[:3])
+        for t in got:
+            assert (t == t[0:1]).all(), f"{name} B={B} L={L} run {rep}: a copy differs from copy 0"
+        if first is None:
+            first = got
+        else:
+            assert all((a == b).all() for a, b in zip(got, first)), f"{name} B={B} L={L}: run {rep} differs from run 0"
+    model.close()
