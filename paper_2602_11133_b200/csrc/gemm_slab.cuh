@@ -514,4 +514,250 @@ gemm_slab_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmW, co
     if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, 4);
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// Gate/up projection + SwiGLU for canvases of 353 .. 384 rows: two units of work per CTA pair, one launch.
+//
+// With S pair-slabs and P pairs on the device (96 and 74 for d_ff = 12288 on 148 SMs) one slab per pair leaves slabs
+// over, and cutting those along K needs a second launch, a reduce-scatter and an epilogue that nothing overlaps.
+// Here A = S - B pairs each take ONE WHOLE slab (all tokens: accumulators of 256 + 128 token columns), and then one of
+// the remaining B = S / 4 slabs for ONE THIRD of the tokens (128 token columns, full K): 3 B <= A second units, no
+// partial sums anywhere.  The second unit's accumulator is a third region of tensor memory (256 + 128 + 128 = 512
+// columns), so the first unit's epilogue runs under the second unit's main loop.  Its four chunk buffers are the last
+// 16 KB of the first four pipeline stages: a second-unit stage holds 16 KB of W and 8 KB of tokens and leaves exactly
+// that much of its 40 KB unused.  Weights of a second-unit slab are read by three pairs, at about the same time: from
+// HBM once.
+constexpr int kSlab2Stages = 5;
+constexpr int kSlab2StageBytes = 128 * 128 + 192 * 128;         // W tile + this CTA's half of 384 tokens
+constexpr int kSlab2Smem = kSlab2Stages * kSlab2StageBytes + 1024;
+
+struct Slab2Plan {
+    int A, B, G;        // pairs (= first units), second-unit slabs, token groups of 128 per second-unit slab
+    bool ok;
+};
+#ifndef JOT_SLAB_TWO_UNITS
+#define JOT_SLAB_TWO_UNITS 1
+#endif
+__host__ __device__ inline Slab2Plan slab2_plan(int M, int n_slabs, int pairs) {
+    Slab2Plan q{0, 0, 3, false};
+    if (!JOT_SLAB_TWO_UNITS) return q;
+    if (M <= 352 || M > 384) return q;             // accumulators of exactly 256 + 128 token columns
+    q.B = n_slabs / (q.G + 1);
+    q.A = n_slabs - q.B;
+    q.ok = q.B > 0 && q.A <= pairs && q.G * q.B <= q.A;
+    return q;
+}
+
+__global__ void __launch_bounds__(kSlabThreads, 1)
+gemm_slab_gateup2_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                         const __grid_constant__ CUtensorMap tmX1) {
+    constexpr int STAGES = kSlab2Stages, STAGE_BYTES = kSlab2StageBytes;
+    constexpr int EPI = SLAB_SWIGLU;          // (for the trace points of instrumented builds)
+    (void)EPI;
+    constexpr int N0 = 256, N1 = 128, H0 = N0 / 2, H1 = N1 / 2;      // token columns per accumulator; rows a CTA loads
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                    // 0 / 1
+    const int pr = (int)(rank & 1u);
+    const bool leader = pr == 0;
+    const int pair = (int)(blockIdx.x >> 1);
+    const int n_slabs = p.N / 256, A = p.slab0, G = p.slab_split, B = n_slabs - A;
+    // unit 0: slab `pair`, every token; unit 1 (pairs below G * B): slab A + pair / G, tokens [128 (pair % G), + 128)
+    const int n_units = pair < G * B ? 2 : 1;
+    const int slab_of[2] = {pair, A + pair / G};
+    const int tok1 = (pair % G) * 128;
+    const int num_kb = (p.K + kBK - 1) / kBK;
+    const int total = n_units * num_kb;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&acc_full[0], 1);
+        mbar_init(&acc_full[1], 1);
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmX);
+        tma_prefetch_desc(&tmX1);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(&tmem_base_slot, 512);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    cluster_sync_all();                       // the pair's barriers exist before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abortp = &abort_flag;
+    if (threadIdx.x == 0) SLAB_TRACE(0);
+    grid_launch_dependents();
+    auto f0_of = [&](int u) { return (2 * slab_of[u] + pr) * 64; };     // first gate row (= output column) of this CTA's tile
+
+    if (warp == 0) {
+        // ================= TMA producer (the whole warp runs the loop, one lane issues) =================
+        const bool elected = elect_one();
+        auto load_w = [&](int stage, int i, uint32_t full_leader) {
+            const int u = i >= num_kb, kb = i - u * num_kb, f0 = f0_of(u);
+            uint8_t* sW = smem + stage * STAGE_BYTES;
+            if (leader) mbar_arrive_expect_tx(&full_bar[stage], u ? 2 * (128 * 128 + H1 * 128) : 2 * STAGE_BYTES);
+            tma_load_2d_pair(sW, &tmW, full_leader, kb * kBK, f0);                          // 64 gate rows
+            tma_load_2d_pair(sW + 64 * 128, &tmW, full_leader, kb * kBK, p.N / 2 + f0);     // the matching 64 up rows
+        };
+        auto load_x = [&](int stage, int i, uint32_t full_leader) {
+            const int u = i >= num_kb, kb = i - u * num_kb;
+            uint8_t* sX = smem + stage * STAGE_BYTES + 128 * 128;
+            if (u == 0) {
+                tma_load_2d_pair(sX, &tmX, full_leader, kb * kBK, pr * H0);
+                tma_load_2d_pair(sX + H0 * 128, &tmX1, full_leader, kb * kBK, N0 + pr * H1);
+            } else {
+                tma_load_2d_pair(sX, &tmX1, full_leader, kb * kBK, tok1 + pr * H1);
+            }
+        };
+        // the first W tiles go out before the wait on the preceding kernel (weights are nobody's output)
+        const int n_pre = min(STAGES, total);
+        if (elected)
+            for (int i = 0; i < n_pre; ++i) load_w(i, i, mapa_u32(&full_bar[i], 0));
+        __syncwarp();
+        grid_dependency_wait();
+        if (lane == 0) SLAB_TRACE(1);
+        if (elected)
+            for (int i = 0; i < n_pre; ++i) load_x(i, i, mapa_u32(&full_bar[i], 0));
+        __syncwarp();
+        int stage = 0;
+        uint32_t phase = 1;                   // the ring has been filled once
+        for (int i = n_pre; i < total; ++i) {
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1, abortp)) break;
+            const uint32_t full_leader = mapa_u32(&full_bar[stage], 0);
+            if (elected) {
+                load_w(stage, i, full_leader);
+                load_x(stage, i, full_leader);
+            }
+            __syncwarp();
+            if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer (even CTA of the pair; the whole warp runs the loop, one lane issues) ======
+        if (leader) {
+            const bool elected = elect_one();
+            const uint32_t idesc0 = umma_idesc_bf16(256, N0), idesc1 = umma_idesc_bf16(256, N1);
+            const uint16_t pair_mask = 0x3u;
+            const uint64_t wd0 = umma_desc_k128(smem_u32(smem));
+            const uint64_t xd0 = wd0 + ((128 * 128) >> 4);
+            constexpr uint32_t stage_units = (uint32_t)STAGE_BYTES >> 4, acc_units = (uint32_t)(H0 * 128) >> 4;
+            int stage = 0;
+            uint32_t phase = 0;
+            uint64_t wd = wd0, xd = xd0;
+            bool ok = true;
+            for (int u = 0; ok && u < n_units; ++u) {
+                uint32_t accum = 0;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[stage], phase, abortp)) { ok = false; break; }
+                    if (u == 0 && kb == 0 && lane == 0) SLAB_TRACE(2);
+                    tc_fence_after();
+                    if (elected) {
+                        if (u == 0) {
+#pragma unroll
+                            for (int k = 0; k < kBK / 16; ++k) {
+                                umma_bf16_pair(tmem_base, wd + 2 * k, xd + 2 * k, idesc0, accum | k);
+                                umma_bf16_pair(tmem_base + N0, wd + 2 * k, xd + acc_units + 2 * k, idesc1, accum | k);
+                            }
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < kBK / 16; ++k)
+                                umma_bf16_pair(tmem_base + N0 + N1, wd + 2 * k, xd + 2 * k, idesc1, accum | k);
+                        }
+                        umma_commit_pair(&empty_bar[stage], pair_mask);
+                    }
+                    __syncwarp();
+                    accum = 1;
+                    wd += stage_units;
+                    xd += stage_units;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; wd = wd0; xd = xd0; }
+                }
+                if (ok && elected) umma_commit_pair(&acc_full[u], pair_mask);
+                __syncwarp();
+                if (lane == 0) SLAB_TRACE(3 + u);
+            }
+        }
+    } else {
+        // ================= epilogue: warps 2..9, two warps per TMEM lane quadrant (a lane is an output FEATURE) =======
+        const int quad = warp & 3, grp = (warp - 2) >> 2;
+        const int f_in = quad * 32 + lane;
+        const uint32_t lane_base = tmem_base + (uint32_t(quad * 32) << 16);
+        // chunk buffer i of the group = bytes [24 KB, 40 KB) of pipeline stage 2 grp + i: free once unit 0's products
+        // have retired (unit 1's loads fill only the first 24 KB of a stage; a pair without a second unit loads nothing)
+        auto chunk_buf = [&](int i) { return reinterpret_cast<float*>(smem + (2 * grp + i) * STAGE_BYTES + 24 * 1024); };
+        const uint32_t bar_id = 1 + grp;
+        const int n_out = p.N / 2;
+        grid_dependency_wait();
+        int it = 0;
+        for (int u = 0; u < n_units; ++u) {
+            // (the tensor-memory loads below are warp-wide: a warp gives up as one)
+            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[u], 0, abortp))) break;
+            tc_fence_after();
+            if (threadIdx.x == 64) SLAB_TRACE(5 + 2 * u);
+            const int f0 = f0_of(u);
+            const int n_ch = u ? N1 / 32 : (N0 + N1) / 32;                    // 32-token chunks of this unit
+            const uint32_t col0 = u ? N0 + N1 : 0;                            // its first accumulator column
+            const int tok0 = u ? tok1 : 0;                                     // its first token
+            float v[32], vn[32];
+            if (grp < n_ch) tmem_ld32(lane_base + col0 + grp * 32, v);
+            tmem_ld_wait_regs(v);
+            for (int c = grp; c < n_ch; c += 2, ++it) {
+                const bool more = c + 2 < n_ch;
+                if (more) tmem_ld32(lane_base + col0 + (c + 2) * 32, vn);     // the next chunk's accumulators travel meanwhile
+                const int t0 = tok0 + c * 32;
+                float* sb = chunk_buf(it & 1);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) sb[j * 128 + f_in] = v[j];
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+                // token-major read-out of the 32 x 128 chunk (64 gate + 64 up features per token), 16-byte stores
+#pragma unroll 1
+                for (int item = f_in; item < 32 * 8; item += 128) {
+                    const int tok = item >> 3, gq = item & 7, t = t0 + tok, oc = f0 + gq * 8;
+                    if (t >= p.M || oc >= n_out) continue;
+                    const float* gp = sb + tok * 128 + gq * 8;
+                    const float4 g0 = *reinterpret_cast<const float4*>(gp), g1 = *reinterpret_cast<const float4*>(gp + 4);
+                    const float4 u0 = *reinterpret_cast<const float4*>(gp + 64), u1 = *reinterpret_cast<const float4*>(gp + 68);
+                    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+                    const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+                    uint4 ov;
+                    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float a0 = gg[2 * j] / (1.f + __expf(-gg[2 * j])) * uu[2 * j];
+                        const float a1 = gg[2 * j + 1] / (1.f + __expf(-gg[2 * j + 1])) * uu[2 * j + 1];
+                        o2[j] = __floats2bfloat162_rn(a0, a1);
+                    }
+                    *reinterpret_cast<uint4*>(p.C + (size_t)t * p.ldc + oc) = ov;
+                }
+                if (more) {
+                    tmem_ld_wait_regs(vn);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = vn[j];
+                }
+            }
+            if (threadIdx.x == 64) SLAB_TRACE(6 + 2 * u);
+        }
+    }
+    __syncwarp();
+
+    // ---- teardown: nobody leaves while the other CTA of the pair may still signal or read across ----
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag && p.status) atomicExch(p.status, 4);
+}
+
 }  // namespace jot

@@ -214,6 +214,35 @@ int launch_slab_t(GemmParams p, const CUtensorMap& tmW, const SlabMaps& tmX, int
     return launch_check();
 }
 
+// Gate/up + SwiGLU for canvases of 353 .. 384 rows: one launch, two units of work per pair (gemm_slab.cuh).
+int launch_slab_gateup2(GemmParams p, const CUtensorMap& tmW, const SlabMaps& tmX, const Slab2Plan& plan, cudaStream_t st) {
+    static thread_local bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev & 63]) {
+        JOT_CUDA(cudaFuncSetAttribute(gemm_slab_gateup2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSlab2Smem));
+        attr_set[dev & 63] = true;
+    }
+    p.slab0 = plan.A;
+    p.slab_split = plan.G;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * plan.A));
+    cfg.blockDim = dim3(kSlabThreads);
+    cfg.dynamicSmemBytes = (size_t)kSlab2Smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaLaunchKernelEx(&cfg, gemm_slab_gateup2_kernel, p, tmW, tmX.x0, tmX.x1);
+    return launch_check();
+}
+
 // How many clusters of `split` pairs the device runs side by side (1 CTA per SM: the kernel takes all shared memory).
 int slab_cluster_capacity(int sms, int split) {
     static thread_local int cap[64][5] = {};
@@ -266,6 +295,10 @@ int run_slab(const DeviceInfo* di, const SlabMaps& tmX, const WeightMaps& w, int
         return launch_slab_t<SLAB_SWIGLU>(p, w.m128, tmX, slab0, n, split, st);
     };
     const int cap1 = slab_cluster_capacity(di->sms, 1);
+    if (epi == EPI_SWIGLU && p.N % 256 == 0) {
+        const Slab2Plan plan = slab2_plan(p.M, n_slabs, cap1);
+        if (plan.ok) return launch_slab_gateup2(p, w.m128, tmX, plan, st);
+    }
     // whole waves of unsplit slabs first; what is left over (or a projection with few slabs) is cut along K so
     // that it still fills the machine
     const int full = n_slabs / cap1 * cap1, rest = n_slabs - full;
@@ -538,7 +571,9 @@ int encode_act_maps(jot_model* m, jot_model::ActMaps* am, int M) {
     JOT_TRY(make_map_2d(m->di, &am->attn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim, 128));
     JOT_TRY(make_map_2d(m->di, &am->act, m->act, M, c.d_ff, c.d_ff, 128));
     am->slab = M <= kSlabPreferTokens;
-    am->slab_gate_up = M > 128 && M <= kSlabGateUpTokens;
+    am->slab_gate_up = (M > 128 && M <= kSlabGateUpTokens) ||
+                       ((2 * c.d_ff) % 256 == 0 &&
+                        slab2_plan(M, 2 * c.d_ff / 256, slab_cluster_capacity(m->di->sms, 1)).ok);
     if (am->slab || am->slab_gate_up) {
         JOT_TRY(make_slab_maps(m->di, &am->xa, m->a, M, c.d_model, c.d_model));
         JOT_TRY(make_slab_maps(m->di, &am->xattn, m->attn, M, c.n_q_heads * c.head_dim, c.n_q_heads * c.head_dim));

@@ -25,6 +25,10 @@ GEOMS = {
     "tiny": inputs.TINY,                                                                  # hd 64, MHA
     "gqa": inputs.ModelGeometry(2, 256, 4, 2, 64, 320, 1032, 1000, 10000.0),              # hd 64, GQA 2:1, odd sizes
     "hd128": inputs.ModelGeometry(2, 256, 2, 1, 128, 704, 2048, 2047, 500000.0),          # hd 128, GQA 2:1
+    # feed-forward widths whose gate/up weights form whole 256-row slabs: at 353 .. 384 canvas rows that projection
+    # runs two units of work per CTA pair (8 slabs: every pair has a second unit; 9 slabs: one pair has none)
+    "ff1024": inputs.ModelGeometry(2, 256, 2, 1, 128, 1024, 2048, 2047, 500000.0),
+    "ff1152": inputs.ModelGeometry(2, 256, 4, 2, 64, 1152, 1032, 1000, 10000.0),
 }
 
 
@@ -42,6 +46,10 @@ def masked_canvas(seed, B, P, G, g, p_mask):
     ("hd128", 1, 64, 192, 0.5),        # 256 rows: the largest canvas on that path, one head per CTA
     ("tiny", 2, 30, 70, 0.6),          # 200 rows, two sequences in one token tile, two heads per CTA
     ("tiny", 1, 8, 24, 1.0),           # 32 rows: the smallest accumulator
+    # gate/up as two units per pair (a whole slab, then a third of the tokens of another one)
+    ("ff1024", 1, 128, 256, 0.5),      # 384 rows
+    ("ff1152", 2, 60, 125, 0.6),       # 370 rows: ragged last token group, two sequences, a pair without a second unit
+    ("ff1024", 1, 100, 253, 0.5),      # 353 rows: the smallest canvas on that path
 ])
 def test_denoise_step_matches_oracle(jot, name, B, P, G, p_mask):
     g = GEOMS[name]
